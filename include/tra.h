@@ -1,0 +1,149 @@
+/*
+ * tra.h — C ABI of the Token Radius Attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * One GPU, one stream per call.  The library allocates device memory only inside
+ * tra_plan_create (plan-owned tables, freed by tra_plan_destroy); every tensor is
+ * owned by the caller.  Unless stated otherwise a pointer is a DEVICE pointer to
+ * contiguous memory, 16-byte aligned.  All calls are asynchronous on `stream`
+ * (a cudaStream_t passed as void*, NULL = default stream) and return a status
+ * code; none of them synchronises the device or throws.
+ *
+ * Token order.  N = T*H*W video tokens.  Every token-indexed array handed to the
+ * four hot calls is in TILE-MAJOR order (Section 3.3, "Flash Radius Mask Kernel":
+ * each H x W frame is cut into tile_h x tile_w tiles, edge tiles clipped; tokens
+ * are listed frame by frame, tile by tile, row-major inside a tile).  A block is
+ * `block` consecutive tile-major positions (Algorithm 1: q = u*b + i, q < N);
+ * NB = ceil(N / block).  tra_tile_major_gather / _scatter move tensors between
+ * raster order (n = (t*H + y)*W + x) and tile-major order.
+ *
+ * Shapes.  Q, K, V, O: bf16 [B, heads, N, head_dim].  entropy, budget, radius,
+ * ridx: [B, heads, N].  block_mask: uint8 [B, heads, NB, NB].  row_ptr: int32
+ * [B*heads*NB + 1]; col_idx: int32 [nnz], key blocks ascending inside a row.
+ */
+#ifndef TRA_H_
+#define TRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define TRA_OK 0
+#define TRA_ERR_INVALID_ARG (-1) /* NULL / misaligned pointer, non-positive size, bad flag     */
+#define TRA_ERR_UNSUPPORTED (-2) /* head_dim, block or grid size outside what the kernels take */
+#define TRA_ERR_CAPACITY (-3)    /* col_idx capacity too small (reported by tra_plan_status)   */
+#define TRA_ERR_CUDA (-4)        /* a CUDA runtime / driver call failed                        */
+#define TRA_ERR_TIMEOUT (-5)     /* a bounded device-side wait expired (reported by tra_plan_status) */
+
+/* plan flags */
+#define TRA_KEEP_DIAGONAL 1u /* force block_mask[u][u] = 1 (a token always sees itself, Eq. 15) */
+
+/* candidate-radius policies for the set R of Eq. 14 when cfg.radii == NULL */
+#define TRA_RADII_EXTENDED 0 /* 0..D (D = ceil(frame diagonal)), then D*exp(gamma*m), m = 1..T-1 */
+#define TRA_RADII_LITERAL 1  /* 0..D and +infinity as the full-support radius                    */
+
+typedef struct tra_plan tra_plan_t; /* opaque: grid geometry, thresholds, count table, block boxes */
+
+typedef struct {
+  int T, H, W;         /* latent grid (Section 2.1); 1 <= T,H,W <= 1023                          */
+  int head_dim;        /* d: 64 or 128                                                          */
+  int block;           /* b of Algorithm 1: 64 or 128 for the attention calls; 16..128 for the   */
+                       /* budget/radius/mask calls                                              */
+  int tile_h, tile_w;  /* tile shape of the tile-major order (Section 3.3)                       */
+  double tau;          /* target attention mass of Eq. 4, in (0, 1]                              */
+  double gamma;        /* temporal decay rate of Eq. 10, >= 0                                    */
+  const double* radii; /* HOST pointer: optional strictly ascending candidate radii; the last    */
+                       /* one must reach full support (may be +inf).  NULL = radius_policy       */
+  int n_radii;
+  int radius_policy;   /* TRA_RADII_* (used when radii == NULL)                                  */
+  unsigned flags;      /* TRA_KEEP_DIAGONAL                                                      */
+} tra_config_t;
+
+/* ---- plan ---------------------------------------------------------------------------- */
+
+/* Builds the plan for one grid / gamma / candidate set on the current device: tile-major
+ * coordinates, the squared-distance thresholds floor(r^2 exp(-2 gamma delta)) of Eq. 15, the
+ * boundary-aware count table C_grid of Eq. 13 for every (token coordinate, candidate) — the
+ * lookup table of Section 3.2 — and per-block bounding boxes (Section 3.3).  Work is enqueued
+ * on `stream`; the call returns after the tables are built (it synchronises that stream).
+ * *out is owned by the caller and released with tra_plan_destroy. */
+int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* stream);
+int tra_plan_destroy(tra_plan_t* plan);
+
+/* Geometry queries (host). */
+int tra_plan_num_tokens(const tra_plan_t* plan);   /* N  */
+int tra_plan_num_blocks(const tra_plan_t* plan);   /* NB */
+int tra_plan_num_radii(const tra_plan_t* plan);    /* |R| */
+/* Copies plan tables to HOST buffers (synchronises): radii[|R|] (double), theta[|R|*T]
+ * (int32, theta[k*T + delta]), coord[N*3] (int32 t,y,x per tile-major position).  Any may be NULL. */
+int tra_plan_tables(const tra_plan_t* plan, double* radii, int32_t* theta, int32_t* coord);
+/* Copies the count table to a HOST buffer uint32 [T*H*W*|R|], indexed ((t*H+y)*W+x)*|R| + k. */
+int tra_plan_count_table(const tra_plan_t* plan, uint32_t* counts);
+
+/* Reads and clears the plan's device status word (synchronises `stream`): TRA_OK, or the
+ * first TRA_ERR_CAPACITY / TRA_ERR_TIMEOUT a kernel of this plan recorded since the last call. */
+int tra_plan_status(tra_plan_t* plan, void* stream);
+
+const char* tra_status_string(int status);
+
+/* ---- layout (Section 3.3: Q, K, V are reordered before attention, O restored after) -- */
+
+/* dst[bh, p, :] = src[bh, raster(p), :] for every tile-major position p.  row_bytes = bytes of
+ * one token row (multiple of 16); n_bh = B*heads.  src and dst must not overlap. */
+int tra_tile_major_gather(const tra_plan_t* plan, const void* src_raster, void* dst_tile_major,
+                          int n_bh, int row_bytes, void* stream);
+/* dst[bh, raster(p), :] = src[bh, p, :] — the inverse. */
+int tra_tile_major_scatter(const tra_plan_t* plan, const void* src_tile_major, void* dst_raster,
+                           int n_bh, int row_bytes, void* stream);
+
+/* ---- the four hot calls ------------------------------------------------------------- */
+
+/* Dense attention of Eq. 1 fused with the attention entropy of Eq. 2, accumulated from the
+ * online-softmax state as in Algorithm 2 (H = m + log l - a/l, nats).
+ *   Q, K, V : bf16 [B, heads, N, head_dim], 128-byte aligned.
+ *   O       : bf16, same shape (written).
+ *   entropy : fp32 [B, heads, N] or NULL (NULL = plain dense attention, no entropy work).
+ *   lse     : fp32 [B, heads, N] or NULL; log sum_j exp(s_ij).
+ *   sm_scale: multiplies q.k; pass 1/sqrt(head_dim) for Eq. 1. */
+int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O,
+                     float* entropy, float* lse, int B, int heads, float sm_scale, void* stream);
+
+/* Entropy -> token budget -> radius (Eq. 8 and Eq. 14; Appendix "Entropy-to-budget-to-radius
+ * lookup"): budget = clamp(ceil(tau * exp(entropy)), 1, N) evaluated in fp64; ridx = index of
+ * the smallest candidate radius whose C_grid at the token's coordinate reaches the budget;
+ * radius = that candidate as fp32 (+inf for an infinite full-support radius).
+ *   entropy: fp32 [B, heads, N];  budget: int32 or NULL;  radius: fp32 or NULL;  ridx: uint16. */
+int tra_budget_radius(const tra_plan_t* plan, const float* entropy, int32_t* budget, float* radius,
+                      uint16_t* ridx, int B, int heads, void* stream);
+
+/* Algorithm 1: block mask from per-query radii.  For every (head, query block u, key block v):
+ * c_j = number of valid queries of u whose disk (Eq. 15) holds key column j; keep the pair iff
+ * some c_j > 0 and 10*#{c_j > b/3} > 6*#{c_j > 0}.  Block bounding boxes only skip pairs whose
+ * vote is already decided; the result equals the unpruned vote bit for bit.
+ *   ridx      : uint16 [B, heads, N] from tra_budget_radius.
+ *   block_mask: uint8 [B, heads, NB, NB] (written, 0/1).
+ *   row_ptr   : int32 [B*heads*NB + 1] (written); col_idx: int32 [col_idx_capacity] (written,
+ *               ascending inside a row).  If nnz exceeds the capacity, col_idx is left partly
+ *               written and TRA_ERR_CAPACITY is recorded in the plan status.
+ *   nnz_out   : device int64 or NULL; total retained blocks. */
+int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* block_mask,
+                         int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
+                         int64_t* nnz_out, int B, int heads, void* stream);
+
+/* Block-sparse attention (Eq. 16 as executed: Section 3.2, last paragraph, and "Limitations"):
+ * softmax attention of each query over all valid keys of the retained key blocks of its block
+ * row; retained blocks are evaluated in full, no token mask inside them.  A query whose block
+ * row is empty gets O = 0.
+ *   row_ptr, col_idx: the CSR list written by tra_build_block_mask (reusable across calls:
+ *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL. */
+int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
+                    const int32_t* row_ptr, const int32_t* col_idx, void* O, float* lse, int B,
+                    int heads, float sm_scale, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TRA_H_ */

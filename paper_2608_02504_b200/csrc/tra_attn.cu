@@ -1,0 +1,730 @@
+// Dense attention with fused entropy (Eq. 1, Eq. 2, Algorithm 2) and block-sparse attention
+// (Eq. 16 as executed over retained blocks) for sm_100a.
+//
+// One CTA owns 256 consecutive query positions of one (batch, head): two 128-row query tiles.
+// Both S = Q K^T and O += P V run on the 5th-generation tensor cores (tcgen05.mma, kind::f16,
+// bf16 operands, fp32 accumulators in tensor memory).  K/V tiles of the retained key blocks are
+// fetched by TMA into a shared-memory ring.  Warp roles:
+//   warps 0-3  softmax of query tile 0 (one thread per query row, tcgen05.ld of its S row)
+//   warps 4-7  softmax of query tile 1
+//   warp  8    TMA producer (Q once, then K_v, V_v for every key block v of the CTA's list)
+//   warp  9    tensor-memory allocation and the single MMA-issuing thread
+// Tensor-memory columns: S0 [0,128)  S1 [128,256)  O0 [256,384)  O1 [384,512); the bf16 P of a
+// tile overwrites the first half of its S columns and feeds the PV MMA straight from tensor memory.
+// The two tiles alternate on the tensor pipe (PV_k(e) then S_k(e+1)) while the other tile's
+// softmax runs.  The key-block list of the CTA is the union of the lists of the query blocks it
+// holds; a tile skips the MMAs of a key block none of its query blocks retains.
+//
+// Online softmax state per row, in the base-2 domain (t = s * sm_scale * log2 e):
+//   m  running reference maximum (raised only when the new maximum exceeds it by more than 8,
+//      so the O accumulator is rescaled rarely; exact because every term uses the same m),
+//   l  = sum 2^(t - m),   a = sum 2^(t - m) (t - m)   (the entropy accumulator of Algorithm 2,
+//      centred on m, which keeps its magnitude small).
+// At the end  O = o / l,  lse = (m + log2 l) ln 2,  H = ln l - ln 2 * a / l
+// (= m + log l - (sum e^(s-m) s) / l of Algorithm 2 with s measured from m).
+//
+// Every wait on an mbarrier is bounded: after about two seconds the waiting thread records
+// TRA_ERR_TIMEOUT in the plan's status word, raises a CTA-wide abort flag and every role leaves
+// its loop; tensor memory is released on every path.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "tra_common.cuh"
+
+namespace {
+
+constexpr int kThreads = 320;
+constexpr int kTileM = 128;           // query rows per tile (UMMA M)
+constexpr int kMaxBitmapWords = 64;   // key blocks per row <= 2048
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kRescaleThreshold = 8.0f;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+// ------------------------------------------------------------------------------------ PTX
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false = gave up (abort flag raised by this or another thread).
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                            int* status) {
+  const unsigned long long t0 = globaltimer_ns();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+        *abort_flag = 1;
+        tra_set_status(status, TRA_ERR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, "
+      "%4}], [%5];" ::"r"(dst),
+      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's tensor-memory lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
+      "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
+      "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() {
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// bf16x2 with `lo` in the low half
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;   // descriptor version
+  d |= 2ull << 61;   // SWIZZLE_128B
+  return d;
+}
+
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, M = 128.
+__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+template <int D, int BN>
+struct Cfg {
+  static constexpr int kGroups = kTileM / BN;                 // query blocks per tile
+  static constexpr int kBlocksPerCta = 2 * kGroups;
+  static constexpr int kQTileBytes = kTileM * D * 2;
+  static constexpr int kSlotBytes = BN * D * 2;
+  static constexpr int kSlots = (D == 128 && BN == 128) ? 5 : 6;
+  static constexpr int kAtoms = D / 64;                        // 64-column swizzle atoms per row
+  static constexpr int kQAtomBytes = kTileM * 128;
+  static constexpr int kKVAtomBytes = BN * 128;
+  static constexpr int kSmemData = 2 * kQTileBytes + kSlots * kSlotBytes;
+  // at least 120 KB so that one CTA owns an SM and its whole tensor memory
+  static constexpr int kSmemNeeded = kSmemData + 1024 /*alignment slack*/ + 2048 /*barriers, bitmaps*/;
+  static constexpr int kSmemBytes = kSmemNeeded > 120 * 1024 ? kSmemNeeded : 120 * 1024;
+};
+
+struct SharedCtl {
+  uint64_t q_full;
+  uint64_t kv_full[6];
+  uint64_t kv_empty[6];
+  uint64_t s_full[2];
+  uint64_t p_ready[2];
+  uint64_t o_done[2];
+  uint64_t drain;
+  uint32_t tmem_base;
+  int abort_flag;
+  uint32_t bitmap[4][kMaxBitmapWords];
+};
+static_assert(sizeof(SharedCtl) <= 2048, "control block");
+
+// ------------------------------------------------------------------------------------ kernel
+template <int D, int BN, bool kEntropy>
+__global__ void __launch_bounds__(kThreads, 1)
+tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ O,
+                float* __restrict__ entropy, float* __restrict__ lse,
+                const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, int N, int NB,
+                float scale_log2, int* __restrict__ status) {
+  using C = Cfg<D, BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;                                   // [2 tiles][atoms][128 rows][64] bf16, swizzled
+  uint8_t* sKV = smem + 2 * C::kQTileBytes;             // ring of K / V tiles
+  SharedCtl* ctl = (SharedCtl*)(smem + C::kSmemData);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int pair = blockIdx.x;
+  const int bh = blockIdx.y;
+  const int q_base = pair * 2 * kTileM;
+  const int n_words = (NB + 31) >> 5;
+  volatile int* abort_flag = &ctl->abort_flag;
+
+  // ---- set-up --------------------------------------------------------------------------
+  if (tid == 0) {
+    mbar_init(smem_u32(&ctl->q_full), 1);
+    for (int i = 0; i < C::kSlots; ++i) {
+      mbar_init(smem_u32(&ctl->kv_full[i]), 1);
+      mbar_init(smem_u32(&ctl->kv_empty[i]), 1);
+    }
+    for (int k = 0; k < 2; ++k) {
+      mbar_init(smem_u32(&ctl->s_full[k]), 1);
+      mbar_init(smem_u32(&ctl->p_ready[k]), kTileM);
+      mbar_init(smem_u32(&ctl->o_done[k]), 1);
+    }
+    mbar_init(smem_u32(&ctl->drain), 1);
+    ctl->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 9) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(
+                     smem_u32(&ctl->tmem_base))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  for (int i = tid; i < 4 * kMaxBitmapWords; i += kThreads) (&ctl->bitmap[0][0])[i] = 0u;
+  __syncthreads();
+  // key-block bitmaps of the query blocks this CTA holds
+  for (int g = 0; g < C::kBlocksPerCta; ++g) {
+    const int ub = pair * C::kBlocksPerCta + g;
+    if (ub >= NB) continue;
+    if (row_ptr == nullptr) {
+      for (int w = tid; w < n_words; w += kThreads) {
+        int rem = NB - 32 * w;
+        ctl->bitmap[g][w] = rem >= 32 ? 0xffffffffu : ((1u << rem) - 1u);
+      }
+    } else {
+      const long long r = (long long)bh * NB + ub;
+      const int lo = row_ptr[r], hi = row_ptr[r + 1];
+      for (int e = lo + tid; e < hi; e += kThreads) {
+        const int v = col_idx[e];
+        if (v >= 0 && v < NB) atomicOr(&ctl->bitmap[g][v >> 5], 1u << (v & 31));
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctl->tmem_base;
+
+  // bitmap of a tile = union over its query blocks
+  auto tile_word = [&](int k, int w) -> uint32_t {
+    uint32_t x = ctl->bitmap[k * C::kGroups][w];
+    if (C::kGroups == 2) x |= ctl->bitmap[k * C::kGroups + 1][w];
+    return x;
+  };
+
+  if (warp == 8) {
+    // ================================================================== TMA producer
+    if (lane == 0) {
+      const uint32_t qbar = smem_u32(&ctl->q_full);
+      mbar_expect_tx(qbar, 2 * C::kQTileBytes);
+      for (int k = 0; k < 2; ++k)
+        for (int a = 0; a < C::kAtoms; ++a)
+          tma_load_3d(smem_u32(sQ + k * C::kQTileBytes + a * C::kQAtomBytes), &map_q, qbar, a * 64,
+                      q_base + k * kTileM, bh);
+      int slot = 0;
+      uint32_t phase = 0;
+      bool alive = true;
+      for (int w = 0; w < n_words && alive; ++w) {
+        uint32_t bits = tile_word(0, w) | tile_word(1, w);
+        while (bits && alive) {
+          const int v = 32 * w + __ffs(bits) - 1;
+          bits &= bits - 1;
+          for (int kv = 0; kv < 2; ++kv) {
+            if (!mbar_wait(smem_u32(&ctl->kv_empty[slot]), phase ^ 1u, abort_flag, status)) {
+              alive = false;
+              break;
+            }
+            const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
+            mbar_expect_tx(fbar, C::kSlotBytes);
+            const CUtensorMap* map = kv == 0 ? &map_k : &map_v;
+            for (int a = 0; a < C::kAtoms; ++a)
+              tma_load_3d(smem_u32(sKV + slot * C::kSlotBytes + a * C::kKVAtomBytes), map, fbar, a * 64,
+                          v * BN, bh);
+            if (++slot == C::kSlots) {
+              slot = 0;
+              phase ^= 1u;
+            }
+          }
+        }
+      }
+    }
+  } else if (warp == 9) {
+    // ================================================================== MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t kIdescQK = make_idesc(BN, false);
+      constexpr uint32_t kIdescPV = make_idesc(D, true);
+      bool alive = mbar_wait(smem_u32(&ctl->q_full), 0u, abort_flag, status);
+      tc_fence_after();
+      int slot = 0;
+      uint32_t phase = 0;
+      uint32_t p_parity[2] = {0u, 0u};
+      uint32_t n_pv[2] = {0u, 0u};
+
+      auto issue_s = [&](int k, int kslot) {
+        const uint32_t qa = smem_u32(sQ + k * C::kQTileBytes);
+        const uint32_t ka = smem_u32(sKV + kslot * C::kSlotBytes);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk) {
+          const uint32_t off_q = (kk >> 2) * C::kQAtomBytes + (kk & 3) * 32;
+          const uint32_t off_k = (kk >> 2) * C::kKVAtomBytes + (kk & 3) * 32;
+          tc_mma_ss(tmem + k * 128, make_desc(qa + off_q, 16, 1024), make_desc(ka + off_k, 16, 1024),
+                    kIdescQK, kk > 0 ? 1u : 0u);
+        }
+        tc_commit(smem_u32(&ctl->s_full[k]));
+      };
+      auto issue_pv = [&](int k, int vslot) {
+        const uint32_t va = smem_u32(sKV + vslot * C::kSlotBytes);
+#pragma unroll
+        for (int kk = 0; kk < BN / 16; ++kk) {
+          tc_mma_ts(tmem + 256 + k * 128, tmem + k * 128 + kk * 8,
+                    make_desc(va + kk * 2048, C::kKVAtomBytes, 1024), kIdescPV,
+                    (n_pv[k] > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(smem_u32(&ctl->o_done[k]));
+        ++n_pv[k];
+      };
+      auto advance = [&]() {
+        if (++slot == C::kSlots) {
+          slot = 0;
+          phase ^= 1u;
+        }
+      };
+
+      // walk the union list with one entry of look-ahead
+      int w = 0;
+      uint32_t bits0 = 0, bits1 = 0;      // remaining bits of the current word, per tile
+      auto next_entry = [&](bool& h0, bool& h1) -> bool {
+        while (true) {
+          const uint32_t u = bits0 | bits1;
+          if (u) {
+            const uint32_t low = u & (0u - u);
+            h0 = (bits0 & low) != 0;
+            h1 = (bits1 & low) != 0;
+            bits0 &= ~low;
+            bits1 &= ~low;
+            return true;
+          }
+          if (w >= n_words) return false;
+          bits0 = tile_word(0, w);
+          bits1 = tile_word(1, w);
+          ++w;
+        }
+      };
+
+      bool h[2], hn[2];
+      bool have = alive && next_entry(h[0], h[1]);
+      if (have) {
+        // first K tile
+        alive = mbar_wait(smem_u32(&ctl->kv_full[slot]), phase, abort_flag, status);
+        if (alive) {
+          tc_fence_after();
+          for (int k = 0; k < 2; ++k)
+            if (h[k]) issue_s(k, slot);
+          tc_commit(smem_u32(&ctl->kv_empty[slot]));
+          advance();
+        }
+      }
+      while (have && alive) {
+        const int vslot = slot;
+        const uint32_t vphase = phase;
+        advance();
+        const int kslot = slot;
+        const uint32_t kphase = phase;
+        const bool have_next = next_entry(hn[0], hn[1]);
+        bool v_ready = false, k_ready = false;
+        for (int k = 0; k < 2 && alive; ++k) {
+          if (h[k]) {
+            if (!v_ready) {
+              alive = mbar_wait(smem_u32(&ctl->kv_full[vslot]), vphase, abort_flag, status);
+              v_ready = true;
+            }
+            if (alive) alive = mbar_wait(smem_u32(&ctl->p_ready[k]), p_parity[k], abort_flag, status);
+            if (!alive) break;
+            p_parity[k] ^= 1u;
+            tc_fence_after();
+            issue_pv(k, vslot);
+          }
+          if (have_next && hn[k]) {
+            if (!k_ready) {
+              alive = mbar_wait(smem_u32(&ctl->kv_full[kslot]), kphase, abort_flag, status);
+              k_ready = true;
+              if (!alive) break;
+              tc_fence_after();
+            }
+            issue_s(k, kslot);
+          }
+        }
+        if (!alive) break;
+        tc_commit(smem_u32(&ctl->kv_empty[vslot]));
+        if (have_next) {
+          tc_commit(smem_u32(&ctl->kv_empty[kslot]));
+          advance();
+        }
+        have = have_next;
+        h[0] = hn[0];
+        h[1] = hn[1];
+      }
+      // make sure every MMA has retired before tensor memory is released
+      tc_commit(smem_u32(&ctl->drain));
+      mbar_wait(smem_u32(&ctl->drain), 0u, abort_flag, status);
+    }
+  } else {
+    // ================================================================== softmax + epilogue
+    const int k = warp >> 2;                         // query tile
+    const int r = tid & (kTileM - 1);                // row inside the tile
+    const int row = q_base + k * kTileM + r;
+    const bool row_valid = row < N;
+    const int g_own = k * C::kGroups + r / BN;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t t_s = tmem + lane_base + k * 128;
+    const uint32_t t_o = tmem + lane_base + 256 + k * 128;
+
+    float m = -INFINITY, l = 0.f, a = 0.f;
+    uint32_t n = 0;               // key blocks this tile has processed
+    uint32_t s_parity = 0;
+    bool alive = true;
+
+    for (int w = 0; w < n_words && alive; ++w) {
+      uint32_t bits = tile_word(k, w);
+      const uint32_t own_bits = ctl->bitmap[g_own][w];
+      while (bits) {
+        const uint32_t low = bits & (0u - bits);
+        bits &= ~low;
+        const int v = 32 * w + __ffs(low) - 1;
+        const bool active = (own_bits & low) != 0;
+        const int col_limit = min(BN, N - v * BN);
+
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl->s_full[k]), s_parity, abort_flag, status))) {
+          alive = false;
+          break;
+        }
+        s_parity ^= 1u;
+        tc_fence_after();
+
+        uint32_t s_bits[BN];
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) tmem_ld32(t_s + c * 32, &s_bits[c * 32]);
+        tmem_wait_ld();
+        float s[BN];
+#pragma unroll
+        for (int j = 0; j < BN; ++j) s[j] = __uint_as_float(s_bits[j]);
+
+        if (col_limit < BN) {
+#pragma unroll
+          for (int j = 0; j < BN; ++j)
+            if (j >= col_limit) s[j] = -1e30f;
+        }
+        float alpha = 1.f;
+        float m_use = 0.f;
+        if (active) {
+          float mx0 = s[0], mx1 = s[1];
+#pragma unroll
+          for (int j = 2; j + 3 < BN; j += 4) {
+            mx0 = fmax3(mx0, s[j], s[j + 1]);
+            mx1 = fmax3(mx1, s[j + 2], s[j + 3]);
+          }
+          mx0 = fmax3(mx0, s[BN - 2], s[BN - 1]);
+          const float m_blk = fmaxf(mx0, mx1) * scale_log2;
+          if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
+            alpha = ex2(m - m_blk);                   // 0 when m = -inf
+            a = l > 0.f ? alpha * (a + (m - m_blk) * l) : 0.f;
+            l *= alpha;
+            m = m_blk;
+          }
+          m_use = m;
+        }
+        // rescale the O accumulator when some row of this warp raised its reference maximum
+        const bool warp_rescale = __any_sync(0xffffffffu, alpha != 1.f) && n > 0;
+        if (warp_rescale) {
+          if (!__all_sync(0xffffffffu,
+                          mbar_wait(smem_u32(&ctl->o_done[k]), (n - 1u) & 1u, abort_flag, status))) {
+            alive = false;
+            break;
+          }
+          tc_fence_after();
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t o[32];
+            tmem_ld32(t_o + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
+            tmem_st32(t_o + c * 32, o);
+          }
+        }
+        // probabilities (relative to m), row sum and entropy accumulator
+        uint32_t pk[BN / 2];
+        if (active) {
+          const float neg_m = -m_use;
+          float l0 = 0.f, l1 = 0.f, a0 = 0.f, a1 = 0.f;
+#pragma unroll
+          for (int j = 0; j < BN; j += 2) {
+            const float t0 = fmaf(s[j], scale_log2, neg_m);
+            const float t1 = fmaf(s[j + 1], scale_log2, neg_m);
+            const float p0 = ex2(t0);
+            const float p1 = ex2(t1);
+            l0 += p0;
+            l1 += p1;
+            if (kEntropy) {
+              a0 = fmaf(p0, t0, a0);
+              a1 = fmaf(p1, t1, a1);
+            }
+            pk[j >> 1] = pack_bf16(p0, p1);
+          }
+          l += l0 + l1;
+          if (kEntropy) a += a0 + a1;
+        } else {
+#pragma unroll
+          for (int j = 0; j < BN / 2; ++j) pk[j] = 0u;
+        }
+#pragma unroll
+        for (int c = 0; c < BN / 64; ++c) tmem_st32(t_s + c * 32, &pk[c * 32]);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&ctl->p_ready[k]));
+        ++n;
+      }
+    }
+
+    // ---- epilogue: O = o / l, entropy, lse ------------------------------------------------
+    if (alive && n > 0)
+      alive = __all_sync(0xffffffffu,
+                         mbar_wait(smem_u32(&ctl->o_done[k]), (n - 1u) & 1u, abort_flag, status));
+    if (alive) {
+      tc_fence_after();
+      const float inv_l = l > 0.f ? 1.f / l : 0.f;
+      __nv_bfloat16* orow = O + ((size_t)bh * N + (row_valid ? row : 0)) * D;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t o_bits[32];
+        float o[32];
+        if (n > 0) {
+          tmem_ld32(t_o + c * 32, o_bits);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(o_bits[j]);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) o[j] = 0.f;
+        }
+        if (row_valid) {
+          uint4* dst = (uint4*)(orow + c * 32);
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) {
+            uint4 val;
+            val.x = pack_bf16(o[q4 * 8 + 0] * inv_l, o[q4 * 8 + 1] * inv_l);
+            val.y = pack_bf16(o[q4 * 8 + 2] * inv_l, o[q4 * 8 + 3] * inv_l);
+            val.z = pack_bf16(o[q4 * 8 + 4] * inv_l, o[q4 * 8 + 5] * inv_l);
+            val.w = pack_bf16(o[q4 * 8 + 6] * inv_l, o[q4 * 8 + 7] * inv_l);
+            dst[q4] = val;
+          }
+        }
+      }
+      if (row_valid) {
+        const size_t idx = (size_t)bh * N + row;
+        if (kEntropy && entropy) entropy[idx] = l > 0.f ? logf(l) - kLn2 * a * inv_l : 0.f;
+        if (lse) lse[idx] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+      }
+    }
+  }
+
+  // ---- teardown ------------------------------------------------------------------------
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 9) {
+    if (ctl->abort_flag) {
+      // let copies and MMAs that were in flight when the CTA gave up land before releasing
+      const unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------------------------ host
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_tiled() {
+  static encode_tiled_fn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (encode_tiled_fn)p;
+  }
+  return fn;
+}
+
+// [B*heads, N, d] bf16 viewed as a 3-D tensor (d innermost); box = 64 columns x `rows` tokens.
+int make_map(CUtensorMap* map, const void* base, int d, int N, long long BH, int rows) {
+  encode_tiled_fn enc = get_encode_tiled();
+  if (!enc) return TRA_ERR_CUDA;
+  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
+  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * (cuuint64_t)N};
+  cuuint32_t box[3] = {64u, (cuuint32_t)rows, 1u};
+  cuuint32_t estr[3] = {1u, 1u, 1u};
+  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? TRA_OK : TRA_ERR_CUDA;
+}
+
+template <int D, int BN, bool kEntropy>
+int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O, float* entropy,
+           float* lse, const int32_t* row_ptr, const int32_t* col_idx, long long BH, float sm_scale,
+           cudaStream_t stream) {
+  using C = Cfg<D, BN>;
+  CUtensorMap mq, mk, mv;
+  int rc;
+  if ((rc = make_map(&mq, Q, D, plan->N, BH, kTileM)) != TRA_OK) return rc;
+  if ((rc = make_map(&mk, K, D, plan->N, BH, BN)) != TRA_OK) return rc;
+  if ((rc = make_map(&mv, V, D, plan->N, BH, BN)) != TRA_OK) return rc;
+  auto kern = tra_attn_kernel<D, BN, kEntropy>;
+  TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
+  const int n_pairs = (plan->N + 2 * kTileM - 1) / (2 * kTileM);
+  dim3 grid((unsigned)n_pairs, (unsigned)BH);
+  kern<<<grid, kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, (__nv_bfloat16*)O, entropy, lse, row_ptr,
+                                                  col_idx, plan->N, plan->NB, sm_scale * kLog2e,
+                                                  plan->d_status);
+  TRA_CUDA_CHECK(cudaGetLastError());
+  return TRA_OK;
+}
+
+int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O,
+                  float* entropy, float* lse, const int32_t* row_ptr, const int32_t* col_idx, int B,
+                  int heads, float sm_scale, void* stream_) {
+  if (!plan || !Q || !K || !V || !O || B < 1 || heads < 1) return TRA_ERR_INVALID_ARG;
+  if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O) & 127) return TRA_ERR_INVALID_ARG;
+  if (!(sm_scale > 0.f)) return TRA_ERR_INVALID_ARG;
+  const long long BH = (long long)B * heads;
+  if (BH > 65535 || plan->NB > 32 * kMaxBitmapWords) return TRA_ERR_UNSUPPORTED;
+  cudaStream_t stream = (cudaStream_t)stream_;
+  const int d = plan->cfg.head_dim, b = plan->cfg.block;
+  const bool ent = entropy != nullptr;
+  if (d == 128 && b == 128)
+    return ent ? launch<128, 128, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
+               : launch<128, 128, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
+  if (d == 64 && b == 64)
+    return ent ? launch<64, 64, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
+               : launch<64, 64, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
+  if (d == 64 && b == 128)
+    return ent ? launch<64, 128, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
+               : launch<64, 128, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
+  if (d == 128 && b == 64)
+    return ent ? launch<128, 64, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
+               : launch<128, 64, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
+  return TRA_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+extern "C" int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
+                                void* O, float* entropy, float* lse, int B, int heads, float sm_scale,
+                                void* stream) {
+  return attn_dispatch(plan, Q, K, V, O, entropy, lse, nullptr, nullptr, B, heads, sm_scale, stream);
+}
+
+extern "C" int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
+                               const int32_t* row_ptr, const int32_t* col_idx, void* O, float* lse, int B,
+                               int heads, float sm_scale, void* stream) {
+  if (!row_ptr || !col_idx) return TRA_ERR_INVALID_ARG;
+  return attn_dispatch(plan, Q, K, V, O, nullptr, lse, row_ptr, col_idx, B, heads, sm_scale, stream);
+}

@@ -1,0 +1,57 @@
+// Shared declarations of the TRA B200 library (internal; the public ABI is include/tra.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tra.h"
+
+#define TRA_MAX_SEG 4       // bounding boxes kept per block
+#define TRA_MAX_T 1024
+
+// A box around a group of tokens of one block: frame range and spatial extent.
+struct tra_box_t {
+  int16_t t0, t1, y0, y1, x0, x1, pad0, pad1;
+};
+static_assert(sizeof(tra_box_t) == 16, "box is one 16-byte load");
+
+struct tra_block_boxes_t {
+  tra_box_t box[TRA_MAX_SEG];
+  int32_t n_box;
+  int32_t pad[3];
+};
+static_assert(sizeof(tra_block_boxes_t) == 80, "block boxes");
+
+struct tra_plan {
+  tra_config_t cfg;
+  int N, NB, n_radii;
+  int device;
+  // host copies
+  double* h_radii;
+  int32_t* h_theta;   // [n_radii][T]
+  int32_t* h_coord;   // [N][3]
+  // device tables
+  uint32_t* d_coord_packed;       // [N]  x | y << 10 | t << 20   per tile-major position
+  int32_t* d_raster_of_pos;       // [N]
+  int32_t* d_theta;               // [n_radii][T]
+  float* d_radii_f32;             // [n_radii]
+  uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)
+  tra_block_boxes_t* d_boxes;     // [NB]
+  int* d_status;                  // device status word
+};
+
+__host__ __device__ inline uint32_t tra_pack_coord(int t, int y, int x) {
+  return (uint32_t)x | ((uint32_t)y << 10) | ((uint32_t)t << 20);
+}
+__host__ __device__ inline int tra_coord_x(uint32_t c) { return (int)(c & 1023u); }
+__host__ __device__ inline int tra_coord_y(uint32_t c) { return (int)((c >> 10) & 1023u); }
+__host__ __device__ inline int tra_coord_t(uint32_t c) { return (int)(c >> 20); }
+
+#define TRA_CUDA_CHECK(expr)                      \
+  do {                                            \
+    cudaError_t _e = (expr);                      \
+    if (_e != cudaSuccess) return TRA_ERR_CUDA;   \
+  } while (0)
+
+// Records the first error code in the plan's device status word.
+__device__ inline void tra_set_status(int* status, int code) { atomicCAS(status, 0, code); }

@@ -1,0 +1,350 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the fp64 oracle
+on the same seeded inputs.  Integer stages are compared bit for bit; entropy and outputs within
+the tolerances stated in tests/common.py."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2608_02504_b200 import workloads
+from tests import common
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda"
+
+
+def api():
+    from paper_2608_02504_b200 import api as _api
+    return _api
+
+
+CFG_TINY = workloads.CONFIGS["tiny"]
+# ragged shapes: N = 210 with b = 64 (last block 18 tokens, last CTA half empty);
+# N = 495 with b = 128 (last block 111 tokens, second CTA's second tile ragged)
+CFG_RAGGED64 = common.small_config(3, 7, 10, heads=3, head_dim=64, block=64, tile_h=4, tile_w=4, seed=78)
+CFG_RAGGED128 = common.small_config(5, 9, 11, heads=2, head_dim=128, block=128, tile_h=4, tile_w=4, seed=79)
+CFG_MID128 = common.small_config(6, 16, 24, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16, seed=80,
+                                 s_lo=0.2, s_hi=5.0)
+SMALL = [CFG_TINY, CFG_RAGGED64, CFG_RAGGED128, CFG_MID128]
+IDS = ["tiny", "ragged64", "ragged128", "mid128"]
+
+
+def make_plan(cfg, **kw):
+    return api().Plan.from_config(cfg, **kw)
+
+
+def tile_major_inputs(cfg, plan, heads=None):
+    Qr, Kr, Vr = workloads.make_qkv(cfg, DEV, heads)
+    return plan.tile_major_gather(Qr), plan.tile_major_gather(Kr), plan.tile_major_gather(Vr)
+
+
+# ----------------------------------------------------------------------------- plan tables
+@pytest.mark.parametrize("cfg", SMALL + [workloads.CONFIGS["wan1.3b-480p"]], ids=IDS + ["wan1.3b"])
+@pytest.mark.parametrize("policy", [0, 1])
+def test_plan_tables_bit_exact(cfg, policy):
+    geo = common.oracle_geometry(cfg, policy)
+    plan = make_plan(cfg, radius_policy=policy)
+    radii, theta, coord = plan.tables()
+    assert plan.N == geo.N and plan.NB == geo.NB
+    assert np.array_equal(radii, geo.radii)
+    assert np.array_equal(theta, geo.theta)
+    assert np.array_equal(coord, geo.coord)
+    assert np.array_equal(plan.count_table(), geo.counts)
+    plan.close()
+
+
+def test_plan_rejects_bad_arguments():
+    a = api()
+    for kw in (dict(head_dim=96), dict(block=8), dict(tau=0.0), dict(gamma=-1.0), dict(T=0),
+               dict(radii=[0.0, 1.0, 2.0]),          # last candidate does not reach full support
+               dict(radii=[0.0, 2.0, 1.0, 1e9])):    # not ascending
+        with pytest.raises(a.TraError):
+            make_plan(CFG_TINY, **kw)
+    p = make_plan(CFG_TINY, radii=[0.0, 1.0, 3.5, float("inf")])
+    assert p.n_radii == 4
+    p.close()
+
+
+# ----------------------------------------------------------------------------- layout
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_tile_major_gather_scatter(cfg):
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    x = torch.randn(2, 3, geo.N, 64, device=DEV).to(torch.bfloat16)
+    g = plan.tile_major_gather(x)
+    ref = x.cpu()[:, :, torch.from_numpy(common.raster_of_pos(geo)).long(), :]
+    assert torch.equal(g.cpu(), ref)
+    assert torch.equal(plan.tile_major_scatter(g), x)
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- budget / radius
+@pytest.mark.parametrize("cfg", SMALL + [workloads.CONFIGS["wan1.3b-480p"]], ids=IDS + ["wan1.3b"])
+def test_budget_radius_bit_exact(cfg):
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    rng = np.random.default_rng(11)
+    heads = 3
+    H = rng.uniform(0.0, math.log(geo.N), (1, heads, geo.N)).astype(np.float32)
+    H[0, 0, :7] = [0.0, math.log(geo.N), 1e-6, 30.0, -1.0, 3.0, math.log(geo.N) - 1e-3]
+    bud_ref, fragile = oracle.budget(H[0], geo.tau, geo.N)
+    ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)
+    budget, radius, ridx = plan.budget_radius(torch.from_numpy(H).to(DEV))
+    ok = ~fragile
+    assert fragile.sum() <= 2                      # elements a one-ulp exp() difference could move
+    assert np.array_equal(budget.cpu().numpy()[0][ok], bud_ref[ok])
+    got_ridx = ridx.cpu().numpy().view(np.uint16)[0]
+    assert np.array_equal(got_ridx[ok], ridx_ref[ok])
+    assert np.array_equal(radius.cpu().numpy()[0][ok], geo.radii[ridx_ref].astype(np.float32)[ok])
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- block mask
+def run_mask(plan, ridx_np):
+    ridx = torch.from_numpy(ridx_np.view(np.int16)).to(DEV)[None]
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    plan.check_status()
+    return mask.cpu().numpy()[0], row_ptr.cpu().numpy(), col_idx.cpu().numpy(), int(nnz.item())
+
+
+def random_ridx(geo, heads, rng, kind):
+    n = geo.radii.size
+    if kind == "uniform":
+        return rng.integers(0, n, (heads, geo.N)).astype(np.uint16)
+    if kind == "small":
+        return rng.integers(0, max(2, n // 8), (heads, geo.N)).astype(np.uint16)
+    if kind == "entropy":        # through the real map, like the pipeline does
+        H = rng.uniform(0.0, math.log(geo.N), (heads, geo.N)).astype(np.float32)
+        bud, _ = oracle.budget(H, geo.tau, geo.N)
+        return oracle.select_radius(bud, geo.coord, geo.H, geo.W, geo.counts)
+    if kind == "blocky":         # whole blocks sharp or diffuse: exercises empty rows and full rows
+        per_block = rng.integers(0, n, (heads, geo.NB))
+        r = np.repeat(per_block, geo.block, axis=1)[:, : geo.N]
+        return r.astype(np.uint16)
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+@pytest.mark.parametrize("kind", ["uniform", "small", "entropy", "blocky"])
+def test_block_mask_bit_exact(cfg, kind):
+    geo = common.oracle_geometry(cfg)
+    heads = 3
+    ridx = random_ridx(geo, heads, np.random.default_rng(12), kind)
+    for flags in (0, api().TRA_KEEP_DIAGONAL):
+        plan = make_plan(cfg, flags=flags)
+        mask, row_ptr, col_idx, nnz = run_mask(plan, ridx)
+        ref = np.stack([oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx[h],
+                                          keep_diagonal=bool(flags)) for h in range(heads)])
+        assert np.array_equal(mask, ref)
+        rp, ci = oracle.csr_from_block_mask(ref)
+        assert nnz == rp[-1]
+        assert np.array_equal(row_ptr.astype(np.int64), rp)
+        assert np.array_equal(col_idx[:nnz], ci)
+        plan.close()
+
+
+def test_block_mask_capacity_error_is_reported():
+    cfg = CFG_TINY
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    full = np.full((1, geo.N), geo.radii.size - 1, np.uint16)
+    ridx = torch.from_numpy(full.view(np.int16)).to(DEV)[None]
+    small = torch.empty(3, dtype=torch.int32, device=DEV)
+    plan.build_block_mask(ridx, col_idx=small)
+    assert plan.status() == -3          # TRA_ERR_CAPACITY
+    assert plan.status() == 0           # cleared by the read
+    plan.close()
+
+
+def test_block_mask_sampled_rows_wan13b():
+    # full-size integer stage at the 32,760-token shape: GPU over all rows, oracle on sampled rows
+    cfg = workloads.CONFIGS["wan1.3b-480p"]
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    rng = np.random.default_rng(13)
+    heads = 2
+    ridx = random_ridx(geo, heads, rng, "entropy")
+    mask, row_ptr, col_idx, nnz = run_mask(plan, ridx)
+    u_list = np.unique(np.concatenate([[0, 1, geo.NB - 2, geo.NB - 1], rng.integers(0, geo.NB, 12)]))
+    for h in range(heads):
+        ref = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx[h], u_list=u_list)
+        assert np.array_equal(mask[h][u_list], ref)
+    rp, ci = oracle.csr_from_block_mask(mask)      # CSR must be the ascending list of the mask itself
+    assert np.array_equal(row_ptr.astype(np.int64), rp) and np.array_equal(col_idx[:nnz], ci)
+    assert 0.02 < mask.mean() < 0.98
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- dense attention + entropy
+def oracle_dense_rows(cfg, geo, Qb, Kb, Vb, h, rows):
+    return oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows)
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+def test_entropy_attn_all_rows(cfg):
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    O, H, lse = plan.entropy_attn(Q, K, V, want_lse=True)
+    O2, _, _ = plan.entropy_attn(Q, K, V, want_entropy=False)       # plain dense: same output
+    plan.check_status()
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(geo.N)
+    for h in range(cfg["heads"]):
+        ref = oracle_dense_rows(cfg, geo, Qb, Kb, Vb, h, rows)
+        common.assert_output(O[0, h], ref["O"], f"dense head {h}")
+        common.assert_output(O2[0, h], ref["O"], f"dense(no entropy) head {h}")
+        dH = np.abs(H[0, h].cpu().numpy().astype(np.float64) - ref["H_def"])
+        assert dH.max() <= common.ENTROPY_ATOL, dH.max()
+        dl = np.abs(lse[0, h].cpu().numpy().astype(np.float64) - ref["lse"])
+        assert dl.max() <= 1e-3, dl.max()
+    plan.close()
+
+
+def test_entropy_attn_uniform_and_one_hot_rows():
+    # Q = 0 -> uniform attention: H = log N, O = mean of V.  A huge query -> near one-hot: H ~ 0.
+    cfg = CFG_RAGGED128
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    Q[:, 0] = 0
+    Q[:, 1] = K[:, 1] * 40
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    plan.check_status()
+    assert torch.allclose(H[0, 0], torch.full_like(H[0, 0], math.log(geo.N)), atol=1e-4)
+    assert torch.allclose(O[0, 0].float(), V[0, 0].float().mean(0, keepdim=True).expand(geo.N, -1), atol=1e-2)
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    ref = oracle.attention_rows(Qb[1], Kb[1], Vb[1], common.scale_of(cfg), np.arange(geo.N))
+    assert np.abs(H[0, 1].cpu().numpy() - ref["H_def"]).max() <= common.ENTROPY_ATOL
+    common.assert_output(O[0, 1], ref["O"], "one-hot head")
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- sparse attention
+def sparse_case(cfg, ridx_kind, flags=0, seed=14):
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg, flags=flags)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    ridx = random_ridx(geo, cfg["heads"], np.random.default_rng(seed), ridx_kind)
+    ridx_t = torch.from_numpy(ridx.view(np.int16)).to(DEV)[None]
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx_t)
+    O, lse = plan.sparse_attn(Q, K, V, row_ptr, col_idx, want_lse=True)
+    plan.check_status()
+    return geo, plan, (Q, K, V), ridx, mask.cpu().numpy()[0], O, lse
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=IDS)
+@pytest.mark.parametrize("kind", ["entropy", "blocky", "small"])
+def test_sparse_attn_all_rows(cfg, kind):
+    geo, plan, (Q, K, V), ridx, mask, O, lse = sparse_case(cfg, kind)
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(geo.N)
+    n_empty = 0
+    for h in range(cfg["heads"]):
+        ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx[h])
+        assert np.array_equal(mask[h], ref_mask)
+        vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx[h], rows,
+                                  ref_mask[rows // geo.block], 0)
+        ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis)
+        common.assert_output(O[0, h], ref["O"], f"sparse head {h}")
+        empty = ~vis.any(axis=1)
+        n_empty += int(empty.sum())
+        got = O[0, h].float().cpu().numpy()
+        assert np.all(got[empty] == 0)                               # empty block row -> zeros
+        got_lse = lse[0, h].cpu().numpy().astype(np.float64)
+        assert np.all(np.isneginf(got_lse[empty]))
+        assert np.abs(got_lse[~empty] - ref["lse"][~empty]).max() <= 1e-3
+    if kind == "small":
+        assert n_empty > 0                                           # the degenerate case is exercised
+    plan.close()
+
+
+def test_sparse_attn_full_mask_equals_dense():
+    # every block retained: the sparse call reproduces dense attention (full-support radius)
+    cfg = CFG_RAGGED128
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    full = np.full((cfg["heads"], geo.N), geo.radii.size - 1, np.uint16)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(torch.from_numpy(full.view(np.int16)).to(DEV)[None])
+    assert int(nnz.item()) == cfg["heads"] * geo.NB * geo.NB
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    Od, _, _ = plan.entropy_attn(Q, K, V, want_entropy=False)
+    plan.check_status()
+    assert torch.equal(Os, Od)
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- the chained pipeline
+@pytest.mark.parametrize("cfg", [CFG_TINY, CFG_MID128], ids=["tiny", "mid128"])
+def test_pipeline_chained_on_gpu(cfg):
+    """entropy_attn -> budget_radius -> build_block_mask -> sparse_attn with the GPU's own
+    intermediate results; the oracle is fed the GPU's fp32 entropies for the integer stages."""
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    _, H, _ = plan.entropy_attn(Q, K, V)
+    budget, radius, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    O, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    plan.check_status()
+    Hn = H.cpu().numpy()[0]
+    bud_ref, fragile = oracle.budget(Hn, geo.tau, geo.N)
+    assert not fragile.any()
+    ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)
+    assert np.array_equal(budget.cpu().numpy()[0], bud_ref)
+    assert np.array_equal(ridx.cpu().numpy().view(np.uint16)[0], ridx_ref)
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(geo.N)
+    density = []
+    for h in range(cfg["heads"]):
+        ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx_ref[h])
+        assert np.array_equal(mask.cpu().numpy()[0, h], ref_mask)
+        density.append(ref_mask.mean())
+        vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_ref[h], rows,
+                                  ref_mask[rows // geo.block], 0)
+        ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis)
+        common.assert_output(O[0, h], ref["O"], f"pipeline head {h}")
+        # the entropy the GPU produced is the oracle's, within tolerance
+        dense = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows)
+        assert np.abs(Hn[h] - dense["H_def"]).max() <= common.ENTROPY_ATOL
+    assert 0.0 < np.mean(density) <= 1.0
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- full-size sampled parity
+@pytest.mark.parametrize("name", ["wan1.3b-480p"])
+def test_full_size_sampled_rows(name):
+    """At a BASELINE shape (all heads resident, the launch configuration the benchmark times):
+    sampled (head, row) pairs of dense attention + entropy and of sparse attention."""
+    cfg = workloads.CONFIGS[name]
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    budget, radius, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    plan.check_status()
+    rng = np.random.default_rng(15)
+    ridx_np = ridx.cpu().numpy().view(np.uint16)[0]
+    for h in (0, cfg["heads"] - 1):
+        rows = np.unique(np.concatenate([[0, 127, 128, geo.N - 1, geo.N - 121, 255 * 128 - 1],
+                                         rng.integers(0, geo.N, 26)])).astype(np.int32)
+        Qb, Kb, Vb = (workloads.bf16_bits(x[0, h]) for x in (Q, K, V))
+        ref = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows)
+        common.assert_output(O[0, h][torch.from_numpy(rows).long().to(DEV)], ref["O"], f"dense {name} h{h}")
+        dH = np.abs(H[0, h].cpu().numpy()[rows] - ref["H_def"])
+        assert dH.max() <= common.ENTROPY_ATOL, dH.max()
+        u_list = np.unique(rows // geo.block)
+        ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx_np[h], u_list=u_list)
+        got_mask = mask[0, h].cpu().numpy()[u_list]
+        assert np.array_equal(got_mask, ref_mask)
+        block_rows = ref_mask[np.searchsorted(u_list, rows // geo.block)]
+        vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np[h], rows, block_rows, 0)
+        refs = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis)
+        common.assert_output(Os[0, h][torch.from_numpy(rows).long().to(DEV)], refs["O"], f"sparse {name} h{h}")
+    plan.close()
