@@ -106,7 +106,9 @@ int tra_tile_major_scatter(const tra_plan_t* plan, const void* src_tile_major, v
  *   Q, K, V : bf16 [B, heads, N, head_dim], 128-byte aligned.
  *   O       : bf16, same shape (written).
  *   entropy : fp32 [B, heads, N] or NULL (NULL = plain dense attention, no entropy work).
- *   lse     : fp32 [B, heads, N] or NULL; log sum_j exp(s_ij).
+ *   lse     : fp32 [B, heads, N] or NULL; log sum_j exp(s_ij).  Exact to fp32 rounding when
+ *             entropy is requested; otherwise formed from the bf16-rounded probabilities
+ *             (absolute error up to about 4e-3).
  *   sm_scale: multiplies q.k; pass 1/sqrt(head_dim) for Eq. 1. */
 int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O,
                      float* entropy, float* lse, int B, int heads, float sm_scale, void* stream);
@@ -138,7 +140,8 @@ int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* 
  * row; retained blocks are evaluated in full, no token mask inside them.  A query whose block
  * row is empty gets O = 0.
  *   row_ptr, col_idx: the CSR list written by tra_build_block_mask (reusable across calls:
- *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL. */
+ *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL, -inf for an empty
+ *   row; formed from the bf16-rounded probabilities (absolute error up to about 4e-3). */
 int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
                     const int32_t* row_ptr, const int32_t* col_idx, void* O, float* lse, int B,
                     int heads, float sm_scale, void* stream);

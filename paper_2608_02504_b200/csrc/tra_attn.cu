@@ -473,6 +473,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     const uint32_t t_o = tmem + lane_base + 256 + k * 128;
 
     float m = -INFINITY, l = 0.f, a = 0.f;
+    float l_exact = 0.f;          // unrounded row sum (entropy kernels only)
     uint32_t n = 0;               // key blocks this tile has processed
     uint32_t s_parity = 0;
     bool alive = true;
@@ -520,8 +521,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const float m_blk = fmaxf(mx0, mx1) * scale_log2;
           if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
             alpha = ex2(m - m_blk);                   // 0 when m = -inf
-            a = l > 0.f ? alpha * (a + (m - m_blk) * l) : 0.f;
+            a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
             l *= alpha;
+            l_exact *= alpha;
             m = m_blk;
           }
           m_use = m;
@@ -549,23 +551,30 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         uint32_t pk[BN / 2];
         if (active) {
           const float neg_m = -m_use;
-          float l0 = 0.f, l1 = 0.f, a0 = 0.f, a1 = 0.f;
+          float l0 = 0.f, l1 = 0.f, a0 = 0.f, a1 = 0.f, e0 = 0.f, e1 = 0.f;
 #pragma unroll
           for (int j = 0; j < BN; j += 2) {
             const float t0 = fmaf(s[j], scale_log2, neg_m);
             const float t1 = fmaf(s[j + 1], scale_log2, neg_m);
-            const float p0 = ex2(t0);
-            const float p1 = ex2(t1);
-            l0 += p0;
-            l1 += p1;
-            if (kEntropy) {
-              a0 = fmaf(p0, t0, a0);
-              a1 = fmaf(p1, t1, a1);
+            const float x0 = ex2(t0), x1 = ex2(t1);
+            // the row sum that normalises O uses the bf16-rounded probabilities the PV MMA
+            // consumes, so numerator and denominator of O = (sum p v) / (sum p) agree
+            const uint32_t packed = pack_bf16(x0, x1);
+            l0 += __uint_as_float(packed << 16);
+            l1 += __uint_as_float(packed & 0xffff0000u);
+            if (kEntropy) {               // entropy and lse from the unrounded terms
+              e0 += x0;
+              e1 += x1;
+              a0 = fmaf(x0, t0, a0);
+              a1 = fmaf(x1, t1, a1);
             }
-            pk[j >> 1] = pack_bf16(p0, p1);
+            pk[j >> 1] = packed;
           }
           l += l0 + l1;
-          if (kEntropy) a += a0 + a1;
+          if (kEntropy) {
+            a += a0 + a1;
+            l_exact += e0 + e1;
+          }
         } else {
 #pragma unroll
           for (int j = 0; j < BN / 2; ++j) pk[j] = 0u;
@@ -615,8 +624,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       }
       if (row_valid) {
         const size_t idx = (size_t)bh * N + row;
-        if (kEntropy && entropy) entropy[idx] = l > 0.f ? logf(l) - kLn2 * a * inv_l : 0.f;
-        if (lse) lse[idx] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+        const float l_out = kEntropy ? l_exact : l;
+        if (kEntropy && entropy) entropy[idx] = l_out > 0.f ? logf(l_out) - kLn2 * a / l_out : 0.f;
+        if (lse) lse[idx] = l_out > 0.f ? (m + log2f(l_out)) * kLn2 : -INFINITY;
       }
     }
   }
