@@ -158,8 +158,28 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
       "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
       : "memory");
 }
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Same wait, naming the 32 destination registers of a tcgen05.ld as read-write operands so that
+// the compiler cannot move a use of them above the wait.
+__device__ __forceinline__ void tmem_wait_ld(uint32_t* r) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+                 "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
+                 "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
+                 "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
+                 "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() {
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -461,7 +481,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       tc_commit(smem_u32(&ctl->drain));
       mbar_wait(smem_u32(&ctl->drain), 0u, abort_flag, status);
     }
-  } else {
+  } else if (warp < 8) {
     // ================================================================== softmax + epilogue
     const int k = warp >> 2;                         // query tile
     const int r = tid & (kTileM - 1);                // row inside the tile
@@ -495,38 +515,48 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         s_parity ^= 1u;
         tc_fence_after();
 
-        uint32_t s_bits[BN];
-#pragma unroll
-        for (int c = 0; c < BN / 32; ++c) tmem_ld32(t_s + c * 32, &s_bits[c * 32]);
-        tmem_wait_ld();
-        float s[BN];
-#pragma unroll
-        for (int j = 0; j < BN; ++j) s[j] = __uint_as_float(s_bits[j]);
+        // The S row is streamed from tensor memory in 32-column chunks, twice: once for the row
+        // maximum, once for the probabilities.  The next chunk's load is in flight while the
+        // current one is processed.  P chunk c (16 packed columns) lands on S columns that
+        // chunk c/2 has already delivered.
+        constexpr int kChunks = BN / 32;
+        uint32_t buf[2][32];
+        tmem_ld32(t_s, buf[0]);
+        tmem_wait_ld(buf[0]);
 
-        if (col_limit < BN) {
-#pragma unroll
-          for (int j = 0; j < BN; ++j)
-            if (j >= col_limit) s[j] = -1e30f;
-        }
         float alpha = 1.f;
         float m_use = 0.f;
-        if (active) {
-          float mx0 = s[0], mx1 = s[1];
+        {
+          float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-          for (int j = 2; j + 3 < BN; j += 4) {
-            mx0 = fmax3(mx0, s[j], s[j + 1]);
-            mx1 = fmax3(mx1, s[j + 2], s[j + 3]);
+          for (int c = 0; c < kChunks; ++c) {
+            if (c + 1 < kChunks) tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1) & 1]);
+            else tmem_ld32(t_s, buf[(c + 1) & 1]);          // first chunk again, for the second pass
+            const uint32_t* b = buf[c & 1];
+            if (col_limit >= (c + 1) * 32) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                mx0 = fmax3(mx0, __uint_as_float(b[j]), __uint_as_float(b[j + 1]));
+                mx1 = fmax3(mx1, __uint_as_float(b[j + 2]), __uint_as_float(b[j + 3]));
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c * 32 + j < col_limit) mx0 = fmaxf(mx0, __uint_as_float(b[j]));
+            }
+            tmem_wait_ld(buf[(c + 1) & 1]);
           }
-          mx0 = fmax3(mx0, s[BN - 2], s[BN - 1]);
-          const float m_blk = fmaxf(mx0, mx1) * scale_log2;
-          if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
-            alpha = ex2(m - m_blk);                   // 0 when m = -inf
-            a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
-            l *= alpha;
-            l_exact *= alpha;
-            m = m_blk;
+          if (active) {
+            const float m_blk = fmaxf(mx0, mx1) * scale_log2;
+            if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
+              alpha = ex2(m - m_blk);                   // 0 when m = -inf
+              a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
+              l *= alpha;
+              l_exact *= alpha;
+              m = m_blk;
+            }
+            m_use = m;
           }
-          m_use = m;
         }
         // rescale the O accumulator when some row of this warp raised its reference maximum
         const bool warp_rescale = __any_sync(0xffffffffu, alpha != 1.f) && n > 0;
@@ -541,46 +571,72 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
             tmem_ld32(t_o + c * 32, o);
-            tmem_wait_ld();
+            tmem_wait_ld(o);
 #pragma unroll
             for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
             tmem_st32(t_o + c * 32, o);
           }
         }
         // probabilities (relative to m), row sum and entropy accumulator
-        uint32_t pk[BN / 2];
-        if (active) {
+        {
           const float neg_m = -m_use;
           float l0 = 0.f, l1 = 0.f, a0 = 0.f, a1 = 0.f, e0 = 0.f, e1 = 0.f;
 #pragma unroll
-          for (int j = 0; j < BN; j += 2) {
-            const float t0 = fmaf(s[j], scale_log2, neg_m);
-            const float t1 = fmaf(s[j + 1], scale_log2, neg_m);
-            const float x0 = ex2(t0), x1 = ex2(t1);
-            // the row sum that normalises O uses the bf16-rounded probabilities the PV MMA
-            // consumes, so numerator and denominator of O = (sum p v) / (sum p) agree
-            const uint32_t packed = pack_bf16(x0, x1);
-            l0 += __uint_as_float(packed << 16);
-            l1 += __uint_as_float(packed & 0xffff0000u);
-            if (kEntropy) {               // entropy and lse from the unrounded terms
-              e0 += x0;
-              e1 += x1;
-              a0 = fmaf(x0, t0, a0);
-              a1 = fmaf(x1, t1, a1);
+          for (int c = 0; c < kChunks; ++c) {
+            if (c + 1 < kChunks) tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1 + kChunks) & 1]);
+            const uint32_t* b = buf[(c + kChunks) & 1];
+            uint32_t pk[16];
+            const bool full = active && col_limit >= (c + 1) * 32;
+            if (full) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                const float t0 = fmaf(__uint_as_float(b[j]), scale_log2, neg_m);
+                const float t1 = fmaf(__uint_as_float(b[j + 1]), scale_log2, neg_m);
+                const float x0 = ex2(t0), x1 = ex2(t1);
+                // the row sum that normalises O uses the bf16-rounded probabilities the PV MMA
+                // consumes, so numerator and denominator of O = (sum p v) / (sum p) agree
+                const uint32_t packed = pack_bf16(x0, x1);
+                l0 += __uint_as_float(packed << 16);
+                l1 += __uint_as_float(packed & 0xffff0000u);
+                if (kEntropy) {               // entropy and lse from the unrounded terms
+                  e0 += x0;
+                  e1 += x1;
+                  a0 = fmaf(x0, t0, a0);
+                  a1 = fmaf(x1, t1, a1);
+                }
+                pk[j >> 1] = packed;
+              }
+            } else if (active) {              // ragged last key block: columns >= col_limit do not exist
+#pragma unroll
+              for (int j = 0; j < 32; j += 2) {
+                const bool v0 = c * 32 + j < col_limit, v1 = c * 32 + j + 1 < col_limit;
+                const float t0 = v0 ? fmaf(__uint_as_float(b[j]), scale_log2, neg_m) : -1e30f;
+                const float t1 = v1 ? fmaf(__uint_as_float(b[j + 1]), scale_log2, neg_m) : -1e30f;
+                const float x0 = ex2(t0), x1 = ex2(t1);
+                const uint32_t packed = pack_bf16(x0, x1);
+                l0 += __uint_as_float(packed << 16);
+                l1 += __uint_as_float(packed & 0xffff0000u);
+                if (kEntropy) {
+                  e0 += x0;
+                  e1 += x1;
+                  a0 = fmaf(x0, t0, a0);
+                  a1 = fmaf(x1, t1, a1);
+                }
+                pk[j >> 1] = packed;
+              }
+            } else {                          // this row's query block does not retain the key block
+#pragma unroll
+              for (int j = 0; j < 16; ++j) pk[j] = 0u;
             }
-            pk[j >> 1] = packed;
+            if (c + 1 < kChunks) tmem_wait_ld(buf[(c + 1 + kChunks) & 1]);
+            tmem_st16(t_s + c * 16, pk);
           }
           l += l0 + l1;
           if (kEntropy) {
             a += a0 + a1;
             l_exact += e0 + e1;
           }
-        } else {
-#pragma unroll
-          for (int j = 0; j < BN / 2; ++j) pk[j] = 0u;
         }
-#pragma unroll
-        for (int c = 0; c < BN / 64; ++c) tmem_st32(t_s + c * 32, &pk[c * 32]);
         tmem_wait_st();
         tc_fence_before();
         mbar_arrive(smem_u32(&ctl->p_ready[k]));
@@ -602,7 +658,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         float o[32];
         if (n > 0) {
           tmem_ld32(t_o + c * 32, o_bits);
-          tmem_wait_ld();
+          tmem_wait_ld(o_bits);
 #pragma unroll
           for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(o_bits[j]);
         } else {
