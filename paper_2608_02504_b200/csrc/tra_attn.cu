@@ -166,11 +166,8 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
       "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
-__device__ __forceinline__ void tmem_wait_ld() {
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-// Same wait, naming the 32 destination registers of a tcgen05.ld as read-write operands so that
-// the compiler cannot move a use of them above the wait.
+// Waits for this thread's tcgen05.ld; the 32 destination registers are named as read-write
+// operands so that the compiler cannot move a use of them above the wait.
 __device__ __forceinline__ void tmem_wait_ld(uint32_t* r) {
   asm volatile("tcgen05.wait::ld.sync.aligned;"
                : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),

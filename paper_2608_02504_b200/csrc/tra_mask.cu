@@ -5,37 +5,56 @@
 #define TRA_MASK_WARPS (TRA_MASK_THREADS / 32)
 
 // ---------------------------------------------------------------------------------------
-// Vote kernel.  One CTA per (batch*head, query block u).
+// Vote kernel.  One CTA per (batch*head, query block u); one thread per query of the block.
 //
 // The vote keeps (u, v) iff some key column is reached (c_j > 0) and more than 60% of the
-// reached columns are "high" (3*c_j > b).  Let need = floor(b/3) + 1 be the smallest high
-// count and r* the need-th largest candidate index among the valid queries of u; thresholds
-// grow with the candidate index and shrink with the frame distance.  With the boxes of the
-// two blocks (groups of tokens, each with a frame range and a spatial box):
-//   - if for every box pair even r* at the smallest frame distance cannot bridge the smallest
-//     box distance, at most need-1 queries reach anything in v: no high column, vote = 0;
-//   - if for every box pair r* at the largest frame distance covers the largest box distance,
-//     at least `need` queries reach every key of v: every column is high, vote = 1;
-//   - otherwise the b x b token tests are done: one warp per key block, each lane owning up
-//     to four key columns and looping over the queries held in shared memory.
+// reached columns are "high" (3*c_j > b), where c_j counts the queries of u whose disk
+// (Eq. 15) holds key j.  Two exact devices keep the work far below the b*b tests per pair of
+// the algorithm as printed:
+//
+// 1. Box pre-classification.  Let need = floor(b/3) + 1 be the smallest high count and r* the
+//    need-th largest candidate index among the valid queries of u; thresholds grow with the
+//    candidate index and shrink with the frame distance.  With the boxes of the two blocks
+//    (groups of tokens, each with a frame range and a spatial box):
+//      - if for every box pair even r* at the smallest frame distance cannot bridge the
+//        smallest box distance, at most need-1 queries reach anything in v: no high column,
+//        vote = 0;
+//      - if for every box pair r* at the largest frame distance covers the largest box
+//        distance, at least `need` queries reach every key of v: every column is high, vote = 1.
+// 2. Count field.  For a key frame f that still holds an undecided key block, the count
+//    c(y', x') = #{queries i : (x'-x_i)^2 + (y'-y_i)^2 <= theta[ridx_i][|f - t_i|]} is built for
+//    the whole frame at once: a query's disk meets row y' in the x-interval of half-width
+//    floor(sqrt(theta - (y'-y_i)^2)), which adds +1 / -1 to a difference array in shared
+//    memory; a prefix sum along each row turns it into the counts.  Every undecided key block
+//    then reads the counts of its own keys in that frame (c_j by definition) and accumulates
+//    its numbers of reached and of high columns.
 // The outcome equals the unpruned vote bit for bit.
 // ---------------------------------------------------------------------------------------
-template <bool kThetaInSmem>
+__device__ __forceinline__ int tra_isqrt_small(int n) {
+  // floor(sqrt(n)) for 0 <= n < 2^22: sqrt(n + 0.5) stays at least 0.25/sqrt(n) away from every
+  // integer, far more than the error of the approximate square root
+  float r;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"((float)n + 0.5f));
+  return (int)r;
+}
+
 __global__ void __launch_bounds__(TRA_MASK_THREADS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
                       uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int NB,
-                      int b, int T, int n_radii, int keep_diagonal) {
+                      int b, int T, int H, int W, int keep_diagonal) {
   extern __shared__ int32_t s_dyn[];
-  __shared__ int4 s_q[128];            // x, y, t, ridx*T of each valid query of the block
   __shared__ int s_rank_ridx[128];
   __shared__ tra_block_boxes_t s_ubox;
-  __shared__ int s_rstar, s_ntest, s_count;
+  __shared__ int s_rstar, s_count;
 
-  int32_t* s_theta_star = s_dyn;                       // [T]
-  uint16_t* s_test = (uint16_t*)(s_dyn + T);           // [NB] key blocks needing the token tests
-  int32_t* s_theta = s_dyn + T + ((NB + 1) / 2);       // [n_radii*T] when kThetaInSmem
-  const int32_t* th = kThetaInSmem ? s_theta : theta;
+  const int Wp = W + 1;
+  int32_t* s_theta_star = s_dyn;                                   // [T]
+  int32_t* s_frame_needed = s_dyn + T;                             // [T]
+  int32_t* s_diff = s_dyn + 2 * T;                                 // [H * (W + 1)]
+  uint16_t* s_ne = (uint16_t*)(s_diff + H * Wp);                   // [NB] reached columns
+  uint16_t* s_hi = s_ne + NB;                                      // [NB] high columns
+  uint8_t* s_state = (uint8_t*)(s_hi + NB);                        // [NB] 0 / 1 decided, 2 undecided
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x;
@@ -46,42 +65,49 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   const int q0 = u * b;
   const int nq = min(b, N - q0);                       // valid queries of this block
   const int need = b / 3 + 1;
+  const int HW = H * W;
 
-  if (kThetaInSmem)
-    for (int i = tid; i < n_radii * T; i += TRA_MASK_THREADS) s_theta[i] = theta[i];
+  // this thread's query
+  int qx = 0, qy = 0, qt = 0, qr = 0;
   if (tid < nq) {
     uint32_t c = coord_packed[q0 + tid];
-    int r = ridx_h[q0 + tid];
-    s_q[tid] = make_int4(tra_coord_x(c), tra_coord_y(c), tra_coord_t(c), r * T);
-    s_rank_ridx[tid] = r;
+    qx = tra_coord_x(c);
+    qy = tra_coord_y(c);
+    qt = tra_coord_t(c);
+    qr = ridx_h[q0 + tid];
+    s_rank_ridx[tid] = qr;
   }
   if (tid == 0) {
     s_ubox = boxes[u];
-    s_ntest = 0;
     s_count = 0;
     s_rstar = -1;
+  }
+  for (int i = tid; i < T; i += TRA_MASK_THREADS) s_frame_needed[i] = 0;
+  for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
+    s_ne[v] = 0;
+    s_hi[v] = 0;
   }
   __syncthreads();
 
   // r*: the need-th largest candidate index (ties broken by lane order)
   if (tid < nq) {
-    int mine = s_rank_ridx[tid], rank = 0;
+    int rank = 0;
     for (int j = 0; j < nq; ++j) {
       int o = s_rank_ridx[j];
-      rank += (o > mine) || (o == mine && j < tid);
+      rank += (o > qr) || (o == qr && j < tid);
     }
-    if (rank == need - 1) s_rstar = mine;
+    if (rank == need - 1) s_rstar = qr;
   }
   __syncthreads();
   const int rstar = s_rstar;                            // -1: fewer than `need` valid queries
   if (rstar >= 0)
-    for (int i = tid; i < T; i += TRA_MASK_THREADS) s_theta_star[i] = th[rstar * T + i];
+    for (int i = tid; i < T; i += TRA_MASK_THREADS) s_theta_star[i] = theta[rstar * T + i];
   __syncthreads();
 
-  // classify every key block
+  // ---- 1. classify every key block with the boxes -----------------------------------------
   int kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
-    int decided = 0;   // 0 = vote 0, 1 = vote 1, 2 = needs the token tests
+    int decided = 0;   // 0 = vote 0, 1 = vote 1, 2 = undecided
     if (rstar >= 0) {
       tra_block_boxes_t vb = boxes[v];
       bool all_reject = true, all_accept = true;
@@ -102,8 +128,11 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       decided = all_reject ? 0 : (all_accept ? 1 : 2);
     }
     if (keep_diagonal && v == u) decided = 1;
+    s_state[v] = (uint8_t)decided;
     if (decided == 2) {
-      s_test[atomicAdd(&s_ntest, 1)] = (uint16_t)v;
+      // frames this key block has tokens in
+      int f0 = (v * b) / HW, f1 = (min(N, (v + 1) * b) - 1) / HW;
+      for (int f = f0; f <= f1; ++f) s_frame_needed[f] = 1;
     } else {
       mask_row[v] = (uint8_t)decided;
       kept += decided;
@@ -112,44 +141,75 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   if (kept) atomicAdd(&s_count, kept);
   __syncthreads();
 
-  // token tests for the undecided key blocks: warp per key block
-  const int ntest = s_ntest;
-  for (int it = warp; it < ntest; it += TRA_MASK_WARPS) {
-    const int v = s_test[it];
-    int kx[4], ky[4], kt[4], cnt[4];
-    bool kvalid[4];
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      int j = lane + 32 * m;
-      int k = v * b + j;
-      kvalid[m] = (j < b) && (k < N);
-      uint32_t c = kvalid[m] ? coord_packed[k] : 0u;
-      kx[m] = tra_coord_x(c);
-      ky[m] = tra_coord_y(c);
-      kt[m] = tra_coord_t(c);
-      cnt[m] = 0;
-    }
-    for (int i = 0; i < nq; ++i) {
-      const int4 q = s_q[i];
-#pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        int dt = abs(q.z - kt[m]);
-        int dx = q.x - kx[m], dy = q.y - ky[m];
-        cnt[m] += (dx * dx + dy * dy <= th[q.w + dt]) ? 1 : 0;
+  // ---- 2. count field of every frame that holds an undecided key block ---------------------
+  for (int f = 0; f < T; ++f) {
+    if (!s_frame_needed[f]) continue;                   // uniform across the CTA
+    for (int i = tid; i < H * Wp; i += TRA_MASK_THREADS) s_diff[i] = 0;
+    __syncthreads();
+    if (tid < nq) {
+      const int th = __ldg(theta + qr * T + abs(qt - f));
+      const int R = tra_isqrt_small(th);
+      const int ylo = max(0, qy - R), yhi = min(H - 1, qy + R);
+      for (int yy = ylo; yy <= yhi; ++yy) {
+        const int dy = yy - qy;
+        const int w = tra_isqrt_small(th - dy * dy);
+        atomicAdd(&s_diff[yy * Wp + max(0, qx - w)], 1);
+        atomicAdd(&s_diff[yy * Wp + min(W - 1, qx + w) + 1], -1);
       }
     }
-    int nonempty = 0, high = 0;
+    __syncthreads();
+    // prefix sum along x, one warp per row
+    for (int yy = warp; yy < H; yy += TRA_MASK_WARPS) {
+      int carry = 0;
+      for (int x0 = 0; x0 < W; x0 += 32) {
+        const int x = x0 + lane;
+        int val = x < W ? s_diff[yy * Wp + x] : 0;
 #pragma unroll
-    for (int m = 0; m < 4; ++m) {
-      nonempty += __popc(__ballot_sync(0xffffffffu, kvalid[m] && cnt[m] > 0));
-      high += __popc(__ballot_sync(0xffffffffu, kvalid[m] && 3 * cnt[m] > b));
+        for (int off = 1; off < 32; off <<= 1) {
+          int other = __shfl_up_sync(0xffffffffu, val, off);
+          if (lane >= off) val += other;
+        }
+        val += carry;
+        if (x < W) s_diff[yy * Wp + x] = val;
+        carry = __shfl_sync(0xffffffffu, val, 31);
+      }
     }
-    if (lane == 0) {
-      int keep = (nonempty > 0) && (10 * high > 6 * nonempty);
-      mask_row[v] = (uint8_t)keep;
-      if (keep) atomicAdd(&s_count, 1);
+    __syncthreads();
+    // undecided key blocks with tokens in this frame: one warp per block
+    const int p_begin = f * HW, p_end = min(N, (f + 1) * HW);
+    const int v_first = p_begin / b, v_last = (p_end - 1) / b;
+    for (int v = v_first + warp; v <= v_last; v += TRA_MASK_WARPS) {
+      if (s_state[v] != 2) continue;
+      const int ps = max(v * b, p_begin), pe = min((v + 1) * b, p_end);
+      int ne = 0, hi = 0;
+      for (int p0 = ps; p0 < pe; p0 += 32) {
+        const int p = p0 + lane;
+        int c = 0;
+        if (p < pe) {
+          const uint32_t kc = coord_packed[p];
+          c = s_diff[tra_coord_y(kc) * Wp + tra_coord_x(kc)];
+        }
+        ne += __popc(__ballot_sync(0xffffffffu, c > 0));
+        hi += __popc(__ballot_sync(0xffffffffu, 3 * c > b));
+      }
+      if (lane == 0) {            // one warp owns v inside a frame; frames are processed in turn
+        s_ne[v] = (uint16_t)(s_ne[v] + ne);
+        s_hi[v] = (uint16_t)(s_hi[v] + hi);
+      }
     }
+    __syncthreads();
   }
+
+  // ---- 3. votes of the undecided key blocks -------------------------------------------------
+  kept = 0;
+  for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
+    if (s_state[v] != 2) continue;
+    const int ne = s_ne[v], hi = s_hi[v];
+    const int keep = (ne > 0) && (10 * hi > 6 * ne);
+    mask_row[v] = (uint8_t)keep;
+    kept += keep;
+  }
+  if (kept) atomicAdd(&s_count, kept);
   __syncthreads();
   if (tid == 0) row_ptr[bh * NB + u + 1] = s_count;   // per-row count; scanned in place afterwards
 }
@@ -217,31 +277,22 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
       col_idx_capacity < 0)
     return TRA_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)stream_;
-  const int NB = plan->NB, T = plan->cfg.T, nr = plan->n_radii;
+  const int NB = plan->NB, T = plan->cfg.T;
   const long long BH = (long long)B * heads;
   if (NB > 65535 || BH > 65535) return TRA_ERR_UNSUPPORTED;
   const long long rows = BH * NB;
 
-  size_t base_words = (size_t)T + (NB + 1) / 2;
-  size_t smem_with_theta = (base_words + (size_t)nr * T) * sizeof(int32_t);
+  const int H = plan->cfg.H, W = plan->cfg.W;
+  size_t smem = ((size_t)2 * T + (size_t)H * (W + 1)) * sizeof(int32_t) + (size_t)NB * 5;
+  smem = (smem + 15) & ~(size_t)15;
+  if (smem > 200 * 1024) return TRA_ERR_UNSUPPORTED;     // frame too large for the count field
   dim3 grid((unsigned)NB, (unsigned)BH);
-  if (smem_with_theta <= 160 * 1024) {
-    if (smem_with_theta > 48 * 1024)
-      TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_block_vote_kernel<true>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)smem_with_theta));
-    tra_block_vote_kernel<true><<<grid, TRA_MASK_THREADS, smem_with_theta, stream>>>(
-        ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, NB,
-        plan->cfg.block, T, nr, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
-  } else {
-    size_t smem = base_words * sizeof(int32_t);
-    if (smem > 48 * 1024)
-      TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_block_vote_kernel<false>,
-                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    tra_block_vote_kernel<false><<<grid, TRA_MASK_THREADS, smem, stream>>>(
-        ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, NB,
-        plan->cfg.block, T, nr, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
-  }
+  if (smem > 48 * 1024)
+    TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_block_vote_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)smem));
+  tra_block_vote_kernel<<<grid, TRA_MASK_THREADS, smem, stream>>>(
+      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, NB,
+      plan->cfg.block, T, H, W, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,
                                                   plan->d_status);
