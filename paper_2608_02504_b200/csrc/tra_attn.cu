@@ -112,24 +112,28 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                          uint32_t idesc, uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem].  Descriptors arrive as (lo, hi) words so that stepping along K
+// is one 32-bit add on the issuing thread.
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                          uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
                                           uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
@@ -198,15 +202,14 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return d;
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1).
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
-  uint64_t d = 0;
-  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-  d |= 1ull << 46;   // descriptor version
-  d |= 2ull << 61;   // SWIZZLE_128B
-  return d;
+// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1), as two words:
+//   lo = start address >> 4 (14 bits) | leading byte offset >> 4 at bit 16
+//   hi = stride byte offset >> 4 | version 1 at bit 14 | SWIZZLE_128B (2) at bits 29..31
+__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
+  return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
+}
+__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) {
+  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
 }
 
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, M = 128.
@@ -370,27 +373,35 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       uint32_t p_parity[2] = {0u, 0u};
       uint32_t n_pv[2] = {0u, 0u};
 
+      // descriptor words: K-major operands (Q, K) step 32 B per k-step inside a 64-column atom and
+      // one atom (rows * 128 B) every four k-steps; the MN-major V operand steps 16 rows (2048 B)
+      constexpr uint32_t kHi = desc_hi(1024);
+      const uint32_t q_lo[2] = {desc_lo(smem_u32(sQ), 16), desc_lo(smem_u32(sQ + C::kQTileBytes), 16)};
+      const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);
+      const uint32_t v_lo0 = desc_lo(smem_u32(sKV), C::kKVAtomBytes);
+      const uint32_t s_full_bar[2] = {smem_u32(&ctl->s_full[0]), smem_u32(&ctl->s_full[1])};
+      const uint32_t o_done_bar[2] = {smem_u32(&ctl->o_done[0]), smem_u32(&ctl->o_done[1])};
+
       auto issue_s = [&](int k, int kslot) {
-        const uint32_t qa = smem_u32(sQ + k * C::kQTileBytes);
-        const uint32_t ka = smem_u32(sKV + kslot * C::kSlotBytes);
+        const uint32_t qa = q_lo[k];
+        const uint32_t ka = k_lo0 + (uint32_t)kslot * (C::kSlotBytes >> 4);
+        const uint32_t d = tmem + k * 128;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off_q = (kk >> 2) * C::kQAtomBytes + (kk & 3) * 32;
-          const uint32_t off_k = (kk >> 2) * C::kKVAtomBytes + (kk & 3) * 32;
-          tc_mma_ss(tmem + k * 128, make_desc(qa + off_q, 16, 1024), make_desc(ka + off_k, 16, 1024),
-                    kIdescQK, kk > 0 ? 1u : 0u);
+          const uint32_t off_q = ((kk >> 2) * C::kQAtomBytes + (kk & 3) * 32) >> 4;
+          const uint32_t off_k = ((kk >> 2) * C::kKVAtomBytes + (kk & 3) * 32) >> 4;
+          tc_mma_ss(d, qa + off_q, kHi, ka + off_k, kHi, kIdescQK, kk > 0 ? 1u : 0u);
         }
-        tc_commit(smem_u32(&ctl->s_full[k]));
+        tc_commit(s_full_bar[k]);
       };
       auto issue_pv = [&](int k, int vslot) {
-        const uint32_t va = smem_u32(sKV + vslot * C::kSlotBytes);
+        const uint32_t va = v_lo0 + (uint32_t)vslot * (C::kSlotBytes >> 4);
+        const uint32_t d = tmem + 256 + k * 128;
+        const uint32_t pa = tmem + k * 128;
+        tc_mma_ts(d, pa, va, kHi, kIdescPV, n_pv[k] > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 0; kk < BN / 16; ++kk) {
-          tc_mma_ts(tmem + 256 + k * 128, tmem + k * 128 + kk * 8,
-                    make_desc(va + kk * 2048, C::kKVAtomBytes, 1024), kIdescPV,
-                    (n_pv[k] > 0 || kk > 0) ? 1u : 0u);
-        }
-        tc_commit(smem_u32(&ctl->o_done[k]));
+        for (int kk = 1; kk < BN / 16; ++kk) tc_mma_ts(d, pa + kk * 8, va + kk * (2048 >> 4), kHi, kIdescPV, 1u);
+        tc_commit(o_done_bar[k]);
         ++n_pv[k];
       };
       auto advance = [&]() {
