@@ -217,8 +217,10 @@ def run_ours(args):
 
     O_raster = torch.empty_like(Qr)
 
-    for _ in range(args.warmup):
+    for i in range(args.warmup):
         one_step()
+        if i == 0:                      # fail fast if a kernel recorded an error
+            plan.check_status()
     torch.cuda.synchronize()
     plan.check_status()
 
