@@ -9,6 +9,8 @@
 //   warps 4-7  softmax of query tile 1
 //   warp  8    TMA producer (Q once, then K_v, V_v for every key block v of the CTA's list)
 //   warp  9    tensor-memory allocation and the single MMA-issuing thread
+//   warps 10-11 idle: they complete the third warpgroup, whose registers are handed to the softmax
+//              warps with setmaxnreg so that a softmax thread can keep its whole S row in registers
 // Tensor-memory columns: S0 [0,128)  S1 [128,256)  O0 [256,384)  O1 [384,512); the bf16 P of a
 // tile overwrites the first half of its S columns and feeds the PV MMA straight from tensor memory.
 // The two tiles alternate on the tensor pipe (PV_k(e) then S_k(e+1)) while the other tile's
@@ -33,7 +35,9 @@
 
 namespace {
 
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;         // 12 warps: three per SM sub-partition
+constexpr int kRegsSoftmax = 216;     // per-thread registers after setmaxnreg: 2 * 216 + 72 = 3 * 168
+constexpr int kRegsControl = 72;
 constexpr int kTileM = 128;           // query rows per tile (UMMA M)
 constexpr int kMaxBitmapWords = 64;   // key blocks per row <= 2048
 constexpr float kLog2e = 1.4426950408889634f;
@@ -72,7 +76,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait; false = gave up (abort flag raised by this or another thread).
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             int* status) {
   const unsigned long long t0 = globaltimer_ns();
   for (uint32_t it = 1;; ++it) {
@@ -182,6 +186,18 @@ __device__ __forceinline__ void tmem_wait_ld(uint32_t* r) {
                :
                : "memory");
 }
+// Compiler-only fence on 32 registers filled by an earlier tcgen05.ld: keeps their uses below
+// the tcgen05.wait::ld that precedes this statement.
+__device__ __forceinline__ void reg_fence32(uint32_t* r) {
+  asm volatile(""
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
+                 "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
+                 "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
+                 "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
+                 "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
 __device__ __forceinline__ void tmem_wait_st() {
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
@@ -239,7 +255,7 @@ struct SharedCtl {
   uint64_t kv_full[6];
   uint64_t kv_empty[6];
   uint64_t s_full[2];
-  uint64_t p_ready[2];
+  uint64_t p_ready[2][2];   // [tile][64-key half of the block]
   uint64_t o_done[2];
   uint64_t drain;
   uint32_t tmem_base;
@@ -279,7 +295,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     for (int k = 0; k < 2; ++k) {
       mbar_init(smem_u32(&ctl->s_full[k]), 1);
-      mbar_init(smem_u32(&ctl->p_ready[k]), kTileM);
+      mbar_init(smem_u32(&ctl->p_ready[k][0]), kTileM);
+      mbar_init(smem_u32(&ctl->p_ready[k][1]), kTileM);
       mbar_init(smem_u32(&ctl->o_done[k]), 1);
     }
     mbar_init(smem_u32(&ctl->drain), 1);
@@ -325,6 +342,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     return x;
   };
 
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsControl));
   if (warp == 8) {
     // ================================================================== TMA producer
     if (lane == 0) {
@@ -394,15 +413,24 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         }
         tc_commit(s_full_bar[k]);
       };
-      auto issue_pv = [&](int k, int vslot) {
+      // PV in 64-key halves: the first half starts as soon as the softmax has stored the first 32
+      // packed columns of P
+      const uint32_t p_ready_bar = smem_u32(&ctl->p_ready[0][0]);     // [k][half], 8 bytes apart
+      auto issue_pv = [&](int k, int vslot) -> bool {
         const uint32_t va = v_lo0 + (uint32_t)vslot * (C::kSlotBytes >> 4);
         const uint32_t d = tmem + 256 + k * 128;
         const uint32_t pa = tmem + k * 128;
-        tc_mma_ts(d, pa, va, kHi, kIdescPV, n_pv[k] > 0 ? 1u : 0u);
 #pragma unroll
-        for (int kk = 1; kk < BN / 16; ++kk) tc_mma_ts(d, pa + kk * 8, va + kk * (2048 >> 4), kHi, kIdescPV, 1u);
+        for (int half = 0; half < BN / 64; ++half) {
+          if (!mbar_wait(p_ready_bar + (k * 2 + half) * 8, p_parity[k], abort_flag, status)) return false;
+          tc_fence_after();
+#pragma unroll
+          for (int kk = half * 4; kk < half * 4 + 4; ++kk)
+            tc_mma_ts(d, pa + kk * 8, va + kk * (2048 >> 4), kHi, kIdescPV, (n_pv[k] > 0 || kk > 0) ? 1u : 0u);
+        }
         tc_commit(o_done_bar[k]);
         ++n_pv[k];
+        return true;
       };
       auto advance = [&]() {
         if (++slot == C::kSlots) {
@@ -459,11 +487,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               alive = mbar_wait(smem_u32(&ctl->kv_full[vslot]), vphase, abort_flag, status);
               v_ready = true;
             }
-            if (alive) alive = mbar_wait(smem_u32(&ctl->p_ready[k]), p_parity[k], abort_flag, status);
+            if (alive) alive = issue_pv(k, vslot);
             if (!alive) break;
             p_parity[k] ^= 1u;
-            tc_fence_after();
-            issue_pv(k, vslot);
           }
           if (have_next && hn[k]) {
             if (!k_ready) {
@@ -489,7 +515,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       tc_commit(smem_u32(&ctl->drain));
       mbar_wait(smem_u32(&ctl->drain), 0u, abort_flag, status);
     }
-  } else if (warp < 8) {
+  }
+  } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
     // ================================================================== softmax + epilogue
     const int k = warp >> 2;                         // query tile
     const int r = tid & (kTileM - 1);                // row inside the tile
@@ -520,50 +548,37 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           alive = false;
           break;
         }
-        s_parity ^= 1u;
         tc_fence_after();
 
-        // The S row is streamed from tensor memory in 32-column chunks, twice: once for the row
-        // maximum, once for the probabilities.  The next chunk's load is in flight while the
-        // current one is processed.  P chunk c (16 packed columns) lands on S columns that
-        // chunk c/2 has already delivered.
-        constexpr int kChunks = BN / 32;
-        uint32_t buf[2][32];
-        tmem_ld32(t_s, buf[0]);
-        tmem_wait_ld(buf[0]);
+        // the whole S row of this thread, straight into registers (one load latency)
+        uint32_t sb[BN];
+#pragma unroll
+        for (int c = 0; c < BN / 32; ++c) tmem_ld32(t_s + c * 32, &sb[c * 32]);
+        tmem_wait_ld(&sb[0]);
+#pragma unroll
+        for (int c = 1; c < BN / 32; ++c) reg_fence32(&sb[c * 32]);
 
+        if (col_limit < BN) {          // ragged last key block: columns >= col_limit do not exist
+#pragma unroll
+          for (int j = 0; j < BN; ++j)
+            if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
+        }
         float alpha = 1.f;
-        float m_use = 0.f;
-        {
-          float mx0 = -INFINITY, mx1 = -INFINITY;
+        if (active) {
+          float mx0 = __uint_as_float(sb[0]), mx1 = __uint_as_float(sb[1]);
 #pragma unroll
-          for (int c = 0; c < kChunks; ++c) {
-            if (c + 1 < kChunks) tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1) & 1]);
-            else tmem_ld32(t_s, buf[(c + 1) & 1]);          // first chunk again, for the second pass
-            const uint32_t* b = buf[c & 1];
-            if (col_limit >= (c + 1) * 32) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                mx0 = fmax3(mx0, __uint_as_float(b[j]), __uint_as_float(b[j + 1]));
-                mx1 = fmax3(mx1, __uint_as_float(b[j + 2]), __uint_as_float(b[j + 3]));
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c * 32 + j < col_limit) mx0 = fmaxf(mx0, __uint_as_float(b[j]));
-            }
-            tmem_wait_ld(buf[(c + 1) & 1]);
+          for (int j = 2; j + 3 < BN; j += 4) {
+            mx0 = fmax3(mx0, __uint_as_float(sb[j]), __uint_as_float(sb[j + 1]));
+            mx1 = fmax3(mx1, __uint_as_float(sb[j + 2]), __uint_as_float(sb[j + 3]));
           }
-          if (active) {
-            const float m_blk = fmaxf(mx0, mx1) * scale_log2;
-            if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
-              alpha = ex2(m - m_blk);                   // 0 when m = -inf
-              a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
-              l *= alpha;
-              l_exact *= alpha;
-              m = m_blk;
-            }
-            m_use = m;
+          mx0 = fmax3(mx0, __uint_as_float(sb[BN - 2]), __uint_as_float(sb[BN - 1]));
+          const float m_blk = fmaxf(mx0, mx1) * scale_log2;
+          if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
+            alpha = ex2(m - m_blk);                   // 0 when m = -inf
+            a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
+            l *= alpha;
+            l_exact *= alpha;
+            m = m_blk;
           }
         }
         // rescale the O accumulator when some row of this warp raised its reference maximum
@@ -585,21 +600,19 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             tmem_st32(t_o + c * 32, o);
           }
         }
-        // probabilities (relative to m), row sum and entropy accumulator
+        // probabilities (relative to m), row sum and entropy accumulator; P goes back to tensor
+        // memory 32 keys at a time, and each 64-key half is announced to the MMA issuer on its own
         {
-          const float neg_m = -m_use;
+          const float neg_m = active ? -m : 0.f;
           float l0 = 0.f, l1 = 0.f, a0 = 0.f, a1 = 0.f, e0 = 0.f, e1 = 0.f;
 #pragma unroll
-          for (int c = 0; c < kChunks; ++c) {
-            if (c + 1 < kChunks) tmem_ld32(t_s + (c + 1) * 32, buf[(c + 1 + kChunks) & 1]);
-            const uint32_t* b = buf[(c + kChunks) & 1];
+          for (int c = 0; c < BN / 32; ++c) {
             uint32_t pk[16];
-            const bool full = active && col_limit >= (c + 1) * 32;
-            if (full) {
+            if (active) {
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
-                const float t0 = fmaf(__uint_as_float(b[j]), scale_log2, neg_m);
-                const float t1 = fmaf(__uint_as_float(b[j + 1]), scale_log2, neg_m);
+                const float t0 = fmaf(__uint_as_float(sb[c * 32 + j]), scale_log2, neg_m);
+                const float t1 = fmaf(__uint_as_float(sb[c * 32 + j + 1]), scale_log2, neg_m);
                 const float x0 = ex2(t0), x1 = ex2(t1);
                 // the row sum that normalises O uses the bf16-rounded probabilities the PV MMA
                 // consumes, so numerator and denominator of O = (sum p v) / (sum p) agree
@@ -614,30 +627,16 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 }
                 pk[j >> 1] = packed;
               }
-            } else if (active) {              // ragged last key block: columns >= col_limit do not exist
-#pragma unroll
-              for (int j = 0; j < 32; j += 2) {
-                const bool v0 = c * 32 + j < col_limit, v1 = c * 32 + j + 1 < col_limit;
-                const float t0 = v0 ? fmaf(__uint_as_float(b[j]), scale_log2, neg_m) : -1e30f;
-                const float t1 = v1 ? fmaf(__uint_as_float(b[j + 1]), scale_log2, neg_m) : -1e30f;
-                const float x0 = ex2(t0), x1 = ex2(t1);
-                const uint32_t packed = pack_bf16(x0, x1);
-                l0 += __uint_as_float(packed << 16);
-                l1 += __uint_as_float(packed & 0xffff0000u);
-                if (kEntropy) {
-                  e0 += x0;
-                  e1 += x1;
-                  a0 = fmaf(x0, t0, a0);
-                  a1 = fmaf(x1, t1, a1);
-                }
-                pk[j >> 1] = packed;
-              }
             } else {                          // this row's query block does not retain the key block
 #pragma unroll
               for (int j = 0; j < 16; ++j) pk[j] = 0u;
             }
-            if (c + 1 < kChunks) tmem_wait_ld(buf[(c + 1 + kChunks) & 1]);
             tmem_st16(t_s + c * 16, pk);
+            if (c & 1) {                      // a 64-key half of P is complete
+              tmem_wait_st();
+              tc_fence_before();
+              mbar_arrive(smem_u32(&ctl->p_ready[k][c >> 1]));
+            }
           }
           l += l0 + l1;
           if (kEntropy) {
@@ -645,9 +644,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             l_exact += e0 + e1;
           }
         }
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(smem_u32(&ctl->p_ready[k]));
+        s_parity ^= 1u;
         ++n;
       }
     }
