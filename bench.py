@@ -42,9 +42,10 @@ from paper_2608_02504_b200 import workloads
 METRIC = ("TRA hot-path effective TFLOP/s at 75.6K tokens (4*d*computed pairs / time over dense "
           "warm-up+entropy, budget/radius, block mask and block-sparse attention)")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# DRAM bytes per launch of the sparse attention kernel, from the ncu capture summarised in
-# profiles/ (None until a capture has been taken for the current kernel).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes (read + write) per head of one sparse attention launch at the 75.6K-token shape, from
+# the ncu capture of a 4-head case summarised in profiles/attention_kernels_wan14b-720p_4heads.md
+# (234.4 MB + 59.3 MB for 4 heads); traffic grows in proportion to the head count.
+NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (234.363648e6 + 59.300864e6) / 4
 
 
 def load_peaks():
@@ -299,7 +300,8 @@ def run_ours(args):
 
     roofline = {"bound": "tensor", "kernel": "tra_attn_kernel<128,128,false> (block-sparse attention)",
                 "achieved": round(tf_sparse, 2), "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": round(tf_sparse / peak_tf, 4), "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "frac": round(tf_sparse / peak_tf, 4),
+                "traffic": (NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD * heads if args.config == "wan14b-720p" else None),
                 "peak_source": peak_note, "flops_per_launch": 4.0 * d * pairs_sparse,
                 "launch_ms": round(t_sparse * 1e3, 4)}
     roofline_dense = {"bound": "tensor", "kernel": "tra_attn_kernel<128,128,true> (dense attention + entropy)",

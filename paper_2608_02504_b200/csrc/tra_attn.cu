@@ -211,6 +211,25 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
+// ---- packed fp32 pairs (sm_100 f32x2 arithmetic: one instruction for two lanes of a row) ----
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 // bf16x2 with `lo` in the low half
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t d;
@@ -604,26 +623,28 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // memory 32 keys at a time, and each 64-key half is announced to the MMA issuer on its own
         {
           const float neg_m = active ? -m : 0.f;
-          float l0 = 0.f, l1 = 0.f, a0 = 0.f, a1 = 0.f, e0 = 0.f, e1 = 0.f;
+          const uint64_t scale2 = pack2(scale_log2, scale_log2), neg_m2 = pack2(neg_m, neg_m);
+          uint64_t l2 = 0ull, a2 = 0ull, e2 = 0ull;      // pairs of partial sums
 #pragma unroll
           for (int c = 0; c < BN / 32; ++c) {
             uint32_t pk[16];
             if (active) {
 #pragma unroll
               for (int j = 0; j < 32; j += 2) {
-                const float t0 = fmaf(__uint_as_float(sb[c * 32 + j]), scale_log2, neg_m);
-                const float t1 = fmaf(__uint_as_float(sb[c * 32 + j + 1]), scale_log2, neg_m);
-                const float x0 = ex2(t0), x1 = ex2(t1);
+                const uint64_t t2 = ffma2(pack2(__uint_as_float(sb[c * 32 + j]), __uint_as_float(sb[c * 32 + j + 1])),
+                                          scale2, neg_m2);
+                float t0, t1, x0, x1;
+                unpack2(t2, t0, t1);
+                x0 = ex2(t0);
+                x1 = ex2(t1);
                 // the row sum that normalises O uses the bf16-rounded probabilities the PV MMA
                 // consumes, so numerator and denominator of O = (sum p v) / (sum p) agree
                 const uint32_t packed = pack_bf16(x0, x1);
-                l0 += __uint_as_float(packed << 16);
-                l1 += __uint_as_float(packed & 0xffff0000u);
+                l2 = fadd2(l2, pack2(__uint_as_float(packed << 16), __uint_as_float(packed & 0xffff0000u)));
                 if (kEntropy) {               // entropy and lse from the unrounded terms
-                  e0 += x0;
-                  e1 += x1;
-                  a0 = fmaf(x0, t0, a0);
-                  a1 = fmaf(x1, t1, a1);
+                  const uint64_t x2 = pack2(x0, x1);
+                  e2 = fadd2(e2, x2);
+                  a2 = ffma2(x2, t2, a2);
                 }
                 pk[j >> 1] = packed;
               }
@@ -638,10 +659,14 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               mbar_arrive(smem_u32(&ctl->p_ready[k][c >> 1]));
             }
           }
-          l += l0 + l1;
+          float lo, hi;
+          unpack2(l2, lo, hi);
+          l += lo + hi;
           if (kEntropy) {
-            a += a0 + a1;
-            l_exact += e0 + e1;
+            unpack2(a2, lo, hi);
+            a += lo + hi;
+            unpack2(e2, lo, hi);
+            l_exact += lo + hi;
           }
         }
         s_parity ^= 1u;
