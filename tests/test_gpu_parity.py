@@ -317,10 +317,19 @@ def test_pipeline_chained_on_gpu(cfg):
 
 
 # ----------------------------------------------------------------------------- full-size sampled parity
-@pytest.mark.parametrize("name", ["wan1.3b-480p"])
-def test_full_size_sampled_rows(name):
-    """At a BASELINE shape (all heads resident, the launch configuration the benchmark times):
-    sampled (head, row) pairs of dense attention + entropy and of sparse attention."""
+def sampled_rows(geo, rng, n_random):
+    b = geo.block
+    fixed = [0, b - 1, b, 2 * b - 1, 2 * b, geo.N - 1, (geo.NB - 1) * b, (geo.NB - 1) * b - 1,
+             geo.N // 2, geo.N // 2 + 1]
+    return np.unique(np.concatenate([fixed, rng.integers(0, geo.N, n_random)])).astype(np.int32)
+
+
+@pytest.mark.parametrize("name,heads_checked,n_random",
+                         [("wan1.3b-480p", (0, 11), 26), ("wan14b-720p", (0, 39), 22), ("hunyuan-720p", (0, 23), 14)])
+def test_full_size_sampled_rows(name, heads_checked, n_random):
+    """At the BASELINE shapes, all heads resident, in the launch configuration the benchmark times:
+    sampled (head, row) pairs of dense attention + entropy, the integer stages of their block
+    rows, and sparse attention.  Rows cover the first / last blocks and the ragged tail."""
     cfg = workloads.CONFIGS[name]
     geo = common.oracle_geometry(cfg)
     plan = make_plan(cfg)
@@ -331,21 +340,89 @@ def test_full_size_sampled_rows(name):
     Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
     plan.check_status()
     rng = np.random.default_rng(15)
-    ridx_np = ridx.cpu().numpy().view(np.uint16)[0]
-    for h in (0, cfg["heads"] - 1):
-        rows = np.unique(np.concatenate([[0, 127, 128, geo.N - 1, geo.N - 121, 255 * 128 - 1],
-                                         rng.integers(0, geo.N, 26)])).astype(np.int32)
+    for h in heads_checked:
+        rows = sampled_rows(geo, rng, n_random)
+        rows_t = torch.from_numpy(rows).long().to(DEV)
         Qb, Kb, Vb = (workloads.bf16_bits(x[0, h]) for x in (Q, K, V))
         ref = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows)
-        common.assert_output(O[0, h][torch.from_numpy(rows).long().to(DEV)], ref["O"], f"dense {name} h{h}")
-        dH = np.abs(H[0, h].cpu().numpy()[rows] - ref["H_def"])
+        common.assert_output(O[0, h][rows_t], ref["O"], f"dense {name} h{h}")
+        Hn = H[0, h].cpu().numpy()
+        dH = np.abs(Hn[rows] - ref["H_def"])
         assert dH.max() <= common.ENTROPY_ATOL, dH.max()
+        # integer stages of this head, fed with the GPU's fp32 entropies: bit-exact
+        bud_ref, fragile = oracle.budget(Hn[None], geo.tau, geo.N)
+        assert fragile.sum() <= 1
+        ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)[0]
+        ok = ~fragile[0]
+        assert np.array_equal(budget[0, h].cpu().numpy()[ok], bud_ref[0][ok])
+        ridx_np = ridx[0, h].cpu().numpy().view(np.uint16)
+        assert np.array_equal(ridx_np[ok], ridx_ref[ok])
         u_list = np.unique(rows // geo.block)
-        ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx_np[h], u_list=u_list)
-        got_mask = mask[0, h].cpu().numpy()[u_list]
-        assert np.array_equal(got_mask, ref_mask)
+        ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx_np, u_list=u_list)
+        assert np.array_equal(mask[0, h].cpu().numpy()[u_list], ref_mask)
         block_rows = ref_mask[np.searchsorted(u_list, rows // geo.block)]
-        vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np[h], rows, block_rows, 0)
+        vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np, rows, block_rows, 0)
         refs = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis)
-        common.assert_output(Os[0, h][torch.from_numpy(rows).long().to(DEV)], refs["O"], f"sparse {name} h{h}")
+        common.assert_output(Os[0, h][rows_t], refs["O"], f"sparse {name} h{h}")
+    # CSR of every head is the ascending list of the mask the same call wrote
+    m = mask[0].reshape(-1, geo.NB).bool()
+    counts = m.sum(dim=1)
+    assert torch.equal(row_ptr[1:].long() - row_ptr[:-1].long(), counts)
+    assert int(nnz.item()) == int(counts.sum().item())
+    cols = torch.nonzero(m)[:, 1].int()
+    assert torch.equal(col_idx[: cols.numel()], cols)
+    density = float(counts.sum().item()) / (cfg["heads"] * geo.NB * geo.NB)
+    assert 0.02 < density < 0.9, density
+    plan.close()
+
+
+# ----------------------------------------------------------------------------- reuse across steps
+def test_mask_reuse_across_denoising_steps():
+    """Warm-up reuse (Section 3.3): radii and mask of the last dense step serve every later step;
+    the sparse call never writes them, and with drifted Q/K it still equals the oracle under the
+    frozen mask."""
+    cfg = CFG_MID128
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    q_state, k_state = Q.float(), K.float()
+    _, H, _ = plan.entropy_attn(Q, K, V)
+    _, _, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    frozen = [t.clone() for t in (ridx, mask, row_ptr, col_idx)]
+    ridx_np = ridx.cpu().numpy().view(np.uint16)[0]
+    rows = np.arange(geo.N)
+    for step in range(3):
+        workloads.drift_(q_state, step, 5)
+        workloads.drift_(k_state, step, 6)
+        Q.copy_(q_state)
+        K.copy_(k_state)
+        O, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+        plan.check_status()
+        for t, f in zip((ridx, mask, row_ptr, col_idx), frozen):
+            assert torch.equal(t, f)
+        Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+        for h in range(cfg["heads"]):
+            mh = frozen[1][0, h].cpu().numpy()
+            vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np[h], rows,
+                                      mh[rows // geo.block], 0)
+            ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis)
+            common.assert_output(O[0, h], ref["O"], f"step {step} head {h}")
+    plan.close()
+
+
+def test_attention_rejects_bad_arguments():
+    a = api()
+    plan = make_plan(CFG_TINY)
+    Q = torch.zeros(1, 2, plan.N, 64, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(ValueError):
+        plan.entropy_attn(Q[:, :, :-1].contiguous(), Q, Q)          # wrong token count
+    with pytest.raises(ValueError):
+        plan.entropy_attn(Q.float(), Q, Q)                           # wrong dtype
+    with pytest.raises(a.TraError):
+        plan.entropy_attn(Q, Q, Q, sm_scale=0.0)                      # non-positive scale
+    base = torch.zeros(Q.numel() + 8, dtype=torch.bfloat16, device=DEV)
+    misaligned = base[8:].view(Q.shape)                              # 16-byte, not 128-byte aligned
+    with pytest.raises(a.TraError):
+        plan.entropy_attn(misaligned, Q, Q)
     plan.close()
