@@ -343,8 +343,17 @@ def run_ours(args):
     # ---- 50-step denoising-schedule emulation (Q and K drift, mask built once and reused) ----
     schedule = None
     if args.schedule and rank == 0:
-        schedule = run_schedule(cfg, plan, api, dev, (Q, K, V, O_dense, O_tm, H, budget, radius, ridx, mask,
-                                                      row_ptr, col_idx, nnz), n_sched, n_warm)
+        bufs = (Q, K, V, O_dense, O_tm, H, budget, radius, ridx, mask, row_ptr, col_idx, nnz)
+        q_keep, k_keep = Q.clone(), K.clone()
+        schedule = run_schedule(cfg, plan, api, dev, bufs, n_sched, n_warm)
+        schedule["refresh_variants"] = []
+        for every in (10, 5, 2):        # the paper's refresh ablation: never / every 10 / 5 / 2 steps
+            Q.copy_(q_keep)
+            K.copy_(k_keep)
+            schedule["refresh_variants"].append(run_schedule(cfg, plan, api, dev, bufs, n_sched, n_warm, every))
+        Q.copy_(q_keep)
+        K.copy_(k_keep)
+        del q_keep, k_keep
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region --------
     e2e = None
@@ -380,14 +389,17 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_schedule(cfg, plan, api, dev, bufs, n_steps, n_warm):
-    """Steps 0..n_warm-1 dense with entropy; radii and mask from the last of them; the rest sparse."""
+def run_schedule(cfg, plan, api, dev, bufs, n_steps, n_warm, refresh_every=0):
+    """Steps 0..n_warm-1 dense with entropy; radii and mask from the last of them; the rest sparse.
+    refresh_every = k > 0: every k-th step after the warm-up runs dense attention with entropy
+    again and rebuilds radii and mask (the paper's 'entropy and mask refresh' ablation)."""
     Q, K, V, O_dense, O_tm, H, budget, radius, ridx, mask, row_ptr, col_idx, nnz = bufs
     heads = cfg["heads"]
     q_state = Q.float()       # tile-major fp32 state that drifts; V stays fixed
     k_state = K.float()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * n_steps)]
     build_ms = 0.0
+    n_refresh = 0
     eb0, eb1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for step in range(n_steps):
         workloads.drift_(q_state, step, cfg["seed"] + 1)
@@ -395,9 +407,11 @@ def run_schedule(cfg, plan, api, dev, bufs, n_steps, n_warm):
         Q.copy_(q_state)
         K.copy_(k_state)
         ev[2 * step].record()
-        if step < n_warm:
+        refresh = refresh_every > 0 and step > n_warm and (step - n_warm) % refresh_every == 0
+        n_refresh += int(refresh)
+        if step < n_warm or refresh:
             plan.entropy_attn(Q, K, V, O=O_dense, entropy=H)
-            if step == n_warm - 1:
+            if step == n_warm - 1 or refresh:
                 eb0.record()
                 plan.budget_radius(H, budget=budget, radius=radius, ridx=ridx)
                 plan.build_block_mask(ridx, block_mask=mask, row_ptr=row_ptr, col_idx=col_idx, nnz=nnz)
@@ -410,6 +424,9 @@ def run_schedule(cfg, plan, api, dev, bufs, n_steps, n_warm):
     per_step = [ev[2 * s].elapsed_time(ev[2 * s + 1]) for s in range(n_steps)]
     build_ms = eb0.elapsed_time(eb1)
     N, block = plan.N, plan.block
+    if refresh_every > 0:
+        return {"refresh_every": refresh_every, "refresh_steps": n_refresh,
+                "amortised_ms_per_step": round(float(np.sum(per_step)) / n_steps, 3)}
     return {"steps": n_steps, "dense_warmup_steps": n_warm, "sparse_steps": n_steps - n_warm,
             "amortised_ms_per_step": round(float(np.sum(per_step)) / n_steps, 3),
             "dense_step_ms": round(float(np.mean(per_step[: n_warm - 1])), 3),

@@ -41,6 +41,11 @@ extern "C" {
 /* plan flags */
 #define TRA_KEEP_DIAGONAL 1u /* force block_mask[u][u] = 1 (a token always sees itself, Eq. 15) */
 
+/* entropy-to-budget maps */
+#define TRA_BUDGET_UNIFORM 0   /* K = ceil(tau exp(H)): the uniform-support map of Eq. 8 (the paper's choice) */
+#define TRA_BUDGET_LOGNORMAL 1 /* K = ceil(N Phibar(sqrt(2 (log N - H)) - Phi^-1(tau))): Appendix,           */
+                               /* "Entropy-identified Lognormal mapping"                                    */
+
 /* candidate-radius policies for the set R of Eq. 14 when cfg.radii == NULL */
 #define TRA_RADII_EXTENDED 0 /* 0..D (D = ceil(frame diagonal)), then D*exp(gamma*m), m = 1..T-1 */
 #define TRA_RADII_LITERAL 1  /* 0..D and +infinity as the full-support radius                    */
@@ -60,6 +65,7 @@ typedef struct {
   int n_radii;
   int radius_policy;   /* TRA_RADII_* (used when radii == NULL)                                  */
   unsigned flags;      /* TRA_KEEP_DIAGONAL                                                      */
+  int budget_map;      /* TRA_BUDGET_* used by tra_budget_radius                                 */
 } tra_config_t;
 
 /* ---- plan ---------------------------------------------------------------------------- */
@@ -114,7 +120,8 @@ int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const
                      float* entropy, float* lse, int B, int heads, float sm_scale, void* stream);
 
 /* Entropy -> token budget -> radius (Eq. 8 and Eq. 14; Appendix "Entropy-to-budget-to-radius
- * lookup"): budget = clamp(ceil(tau * exp(entropy)), 1, N) evaluated in fp64; ridx = index of
+ * lookup"): budget = clamp(ceil(tau * exp(entropy)), 1, N) evaluated in fp64 (or the lognormal
+ * map of the appendix when the plan was created with TRA_BUDGET_LOGNORMAL); ridx = index of
  * the smallest candidate radius whose C_grid at the token's coordinate reaches the budget;
  * radius = that candidate as fp32 (+inf for an infinite full-support radius).
  *   entropy: fp32 [B, heads, N];  budget: int32 or NULL;  radius: fp32 or NULL;  ridx: uint16. */

@@ -111,6 +111,20 @@ def budget(entropy_f32, tau, N):
     return out, frag.astype(bool)
 
 
+def budget_lognormal(entropy_f32, tau, N):
+    """K = ceil(N * Phibar(sqrt(2 (log N - H)) - Phi^-1(tau))) clamped to [1, N] (Appendix,
+    entropy-identified Lognormal mapping); also the 'fragile' flags."""
+    from statistics import NormalDist
+    z_tau = NormalDist().inv_cdf(tau) if tau < 1.0 else float("inf")
+    e = _c(entropy_f32, np.float32)
+    out = np.empty(e.shape, np.int32)
+    frag = np.empty(e.shape, np.uint8)
+    lib().tra_oracle_budget_lognormal(_ptr(e, ctypes.c_float), ctypes.c_int64(e.size),
+                                      ctypes.c_double(z_tau), N, _ptr(out, ctypes.c_int32),
+                                      _ptr(frag, ctypes.c_uint8))
+    return out, frag.astype(bool)
+
+
 def select_radius(budget_hn, coord, H, W, counts):
     """ridx[h, p] = index of the smallest candidate with C_grid >= K (Eq. 14)."""
     b = _c(budget_hn, np.int32)

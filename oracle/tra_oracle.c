@@ -198,6 +198,34 @@ void tra_oracle_budget(const float* entropy, int64_t n, double tau, int N, int32
 }
 
 /* ------------------------------------------------------------------------- *
+ * Lognormal entropy-to-budget map (Appendix "Distributional Analysis", entropy-
+ * identified Lognormal mapping): sigma = sqrt(2 (log N - H)),
+ * B = Phibar(sigma - Phi^{-1}(tau)), K = ceil(N * B) clamped to [1, N].
+ * z_tau = Phi^{-1}(tau) is passed in (a constant of the configuration);
+ * Phibar(z) = erfc(z / sqrt 2) / 2.  H above log N (rounding) is treated as log N.
+ * fragile[i] = 1 when N*B lies within 1e-11 (relative) of an integer.
+ * ------------------------------------------------------------------------- */
+void tra_oracle_budget_lognormal(const float* entropy, int64_t n, double z_tau, int N,
+                                 int32_t* budget, uint8_t* fragile) {
+  const double logN = log((double)N);
+  for (int64_t i = 0; i < n; ++i) {
+    double gap = logN - (double)entropy[i];
+    if (gap < 0.0) gap = 0.0;
+    double sigma = sqrt(2.0 * gap);
+    double B = 0.5 * erfc((sigma - z_tau) / sqrt(2.0));
+    double v = (double)N * B;
+    double k = ceil(v);
+    if (fragile) {
+      double scale = v > 1.0 ? v : 1.0;
+      fragile[i] = (fabs(v - rint(v)) <= 1e-11 * scale) && (v < (double)N + 1.0);
+    }
+    if (!(k >= 1.0)) k = 1.0;
+    if (k > (double)N) k = (double)N;
+    budget[i] = (int32_t)k;
+  }
+}
+
+/* ------------------------------------------------------------------------- *
  * Radius selection, Eq. 14: the smallest candidate whose grid count reaches
  * the budget.  coord = tile-major coordinates; counts = table above.  The last
  * candidate has count N, so the scan always stops.

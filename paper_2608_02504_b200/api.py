@@ -19,6 +19,8 @@ TRA_OK = 0
 TRA_KEEP_DIAGONAL = 1
 TRA_RADII_EXTENDED = 0
 TRA_RADII_LITERAL = 1
+TRA_BUDGET_UNIFORM = 0
+TRA_BUDGET_LOGNORMAL = 1
 
 EXPORTS = [
     "tra_plan_create", "tra_plan_destroy", "tra_plan_num_tokens", "tra_plan_num_blocks",
@@ -35,7 +37,7 @@ class tra_config_t(ctypes.Structure):
         ("tile_h", ctypes.c_int), ("tile_w", ctypes.c_int),
         ("tau", ctypes.c_double), ("gamma", ctypes.c_double),
         ("radii", ctypes.POINTER(ctypes.c_double)), ("n_radii", ctypes.c_int),
-        ("radius_policy", ctypes.c_int), ("flags", ctypes.c_uint),
+        ("radius_policy", ctypes.c_int), ("flags", ctypes.c_uint), ("budget_map", ctypes.c_int),
     ]
 
 
@@ -95,7 +97,7 @@ class Plan:
     """Owns a ``tra_plan_t`` (geometry, thresholds, count table, block boxes)."""
 
     def __init__(self, T, H, W, head_dim, block, tile_h, tile_w, tau=0.9, gamma=0.6, radii=None,
-                 radius_policy=TRA_RADII_EXTENDED, flags=0, stream=None):
+                 radius_policy=TRA_RADII_EXTENDED, flags=0, budget_map=TRA_BUDGET_UNIFORM, stream=None):
         cfg = tra_config_t()
         cfg.T, cfg.H, cfg.W = T, H, W
         cfg.head_dim, cfg.block, cfg.tile_h, cfg.tile_w = head_dim, block, tile_h, tile_w
@@ -106,7 +108,7 @@ class Plan:
             self._radii_keepalive = arr
             cfg.radii = ctypes.cast(arr, ctypes.POINTER(ctypes.c_double))
             cfg.n_radii = len(radii)
-        cfg.radius_policy, cfg.flags = radius_policy, flags
+        cfg.radius_policy, cfg.flags, cfg.budget_map = radius_policy, flags, budget_map
         self.cfg = cfg
         self._h = ctypes.c_void_p()
         _check(_lib.tra_plan_create(ctypes.byref(self._h), ctypes.byref(cfg), _stream(stream)), "tra_plan_create")

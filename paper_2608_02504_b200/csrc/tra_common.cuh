@@ -26,6 +26,7 @@ struct tra_plan {
   tra_config_t cfg;
   int N, NB, n_radii;
   int device;
+  double z_tau;       // Phi^-1(tau), for the lognormal budget map
   // host copies
   double* h_radii;
   int32_t* h_theta;   // [n_radii][T]

@@ -78,6 +78,18 @@ __global__ void tra_permute_rows_kernel(const int32_t* __restrict__ raster_of_po
 // ---------------------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------------------
+// Phi^-1(p) for p in (0, 1]: bisection on erfc (monotone), to the last bit that matters here.
+static double tra_inverse_normal_cdf(double p) {
+  if (p >= 1.0) return INFINITY;
+  double lo = -40.0, hi = 40.0;
+  for (int it = 0; it < 200; ++it) {
+    double mid = 0.5 * (lo + hi);
+    double cdf = 0.5 * erfc(-mid / sqrt(2.0));
+    if (cdf < p) lo = mid; else hi = mid;
+  }
+  return 0.5 * (lo + hi);
+}
+
 static void tra_plan_free(tra_plan* p) {
   if (!p) return;
   free(p->h_radii);
@@ -104,6 +116,8 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   if (cfg->block < 16 || cfg->block > 128) return TRA_ERR_UNSUPPORTED;
   if (cfg->head_dim != 64 && cfg->head_dim != 128) return TRA_ERR_UNSUPPORTED;
   if ((long long)T * H * W > (1ll << 30)) return TRA_ERR_UNSUPPORTED;
+  if (cfg->budget_map != TRA_BUDGET_UNIFORM && cfg->budget_map != TRA_BUDGET_LOGNORMAL)
+    return TRA_ERR_INVALID_ARG;
 
   tra_plan* p = new tra_plan();
   memset(p, 0, sizeof(*p));
@@ -111,6 +125,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   p->cfg.radii = nullptr;
   p->N = T * H * W;
   p->NB = (p->N + cfg->block - 1) / cfg->block;
+  p->z_tau = tra_inverse_normal_cdf(cfg->tau);
   if (cudaGetDevice(&p->device) != cudaSuccess) {
     delete p;
     return TRA_ERR_CUDA;

@@ -1,7 +1,10 @@
 // Entropy -> budget -> radius (Eq. 8, Eq. 14; Appendix "Entropy-to-budget-to-radius lookup").
+#include <math.h>
+
 #include "tra_common.cuh"
 
-// One thread per (batch*head, token).  The budget is evaluated in fp64 so that the ceiling is
+// One thread per (batch*head, token).  The budget (uniform-support map of Eq. 8, or the lognormal
+// map of the appendix) is evaluated in fp64 so that the ceiling is
 // taken on the same number a host fp64 evaluation sees; the radius is the first entry of the
 // token's count-table row that reaches the budget (the row is non-decreasing in the candidate
 // index, so a binary search finds the minimum of Eq. 14).
@@ -11,11 +14,19 @@ __global__ void tra_budget_radius_kernel(const float* __restrict__ entropy,
                                          const float* __restrict__ radii, int32_t* __restrict__ budget,
                                          float* __restrict__ radius, uint16_t* __restrict__ ridx,
                                          int N, int H, int W, int n_radii, double tau,
-                                         long long total) {
+                                         int budget_map, double z_tau, double log_n, long long total) {
   long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= total) return;
   int p = (int)(g % N);
-  double v = ceil(tau * exp((double)entropy[g]));
+  double v;
+  if (budget_map == TRA_BUDGET_LOGNORMAL) {
+    // sigma = sqrt(2 (log N - H)),  B = Phibar(sigma - Phi^-1(tau)),  K = ceil(N B)
+    double gap = log_n - (double)entropy[g];
+    if (gap < 0.0) gap = 0.0;
+    v = ceil((double)N * 0.5 * erfc((sqrt(2.0 * gap) - z_tau) * 0.70710678118654752440));
+  } else {
+    v = ceil(tau * exp((double)entropy[g]));
+  }
   if (!(v >= 1.0)) v = 1.0;          // also catches NaN
   if (v > (double)N) v = (double)N;
   uint32_t need = (uint32_t)v;
@@ -41,7 +52,8 @@ extern "C" int tra_budget_radius(const tra_plan_t* plan, const float* entropy, i
   if (grid > 0x7fffffffll) return TRA_ERR_UNSUPPORTED;
   tra_budget_radius_kernel<<<(unsigned)grid, 256, 0, stream>>>(
       entropy, plan->d_coord_packed, plan->d_counts, plan->d_radii_f32, budget, radius, ridx,
-      plan->N, plan->cfg.H, plan->cfg.W, plan->n_radii, plan->cfg.tau, total);
+      plan->N, plan->cfg.H, plan->cfg.W, plan->n_radii, plan->cfg.tau, plan->cfg.budget_map, plan->z_tau,
+      log((double)plan->N), total);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }

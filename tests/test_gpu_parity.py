@@ -102,6 +102,25 @@ def test_budget_radius_bit_exact(cfg):
     plan.close()
 
 
+@pytest.mark.parametrize("cfg", [CFG_TINY, workloads.CONFIGS["wan1.3b-480p"]], ids=["tiny", "wan1.3b"])
+def test_budget_radius_lognormal_map_bit_exact(cfg):
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg, budget_map=api().TRA_BUDGET_LOGNORMAL)
+    rng = np.random.default_rng(21)
+    H = rng.uniform(0.0, math.log(geo.N), (1, 2, geo.N)).astype(np.float32)
+    H[0, 0, :4] = [0.0, math.log(geo.N), 30.0, 1e-3]
+    bud_ref, fragile = oracle.budget_lognormal(H[0], geo.tau, geo.N)
+    ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)
+    budget, radius, ridx = plan.budget_radius(torch.from_numpy(H).to(DEV))
+    ok = ~fragile
+    assert fragile.sum() <= 2
+    assert np.array_equal(budget.cpu().numpy()[0][ok], bud_ref[ok])
+    assert np.array_equal(ridx.cpu().numpy().view(np.uint16)[0][ok], ridx_ref[ok])
+    plan.close()
+    with pytest.raises(api().TraError):
+        make_plan(cfg, budget_map=7)
+
+
 # ----------------------------------------------------------------------------- block mask
 def run_mask(plan, ridx_np):
     ridx = torch.from_numpy(ridx_np.view(np.int16)).to(DEV)[None]

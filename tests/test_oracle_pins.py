@@ -132,6 +132,33 @@ def test_budget_closed_forms_and_monotone():
     assert fr[0]
 
 
+def test_budget_lognormal_closed_forms():
+    # Appendix, entropy-identified Lognormal mapping: sigma = sqrt(2 (ln N - H)),
+    # B = Phibar(sigma - Phi^-1(tau)); scipy's norm.sf / norm.ppf are the library routines.
+    import scipy.stats
+    N, tau = 75600, 0.9
+    H = np.array([math.log(N), 0.0, 5.0, 9.0, 10.5, 11.0], np.float32)
+    b, _ = oracle.budget_lognormal(H, tau, N)
+    # sigma = 0 at H = ln N: B = Phibar(-z_tau) = tau (the uniform map's value there)
+    # (fp32 ln N is a hair below ln N and dB/dsigma is steep at 0, hence the small slack)
+    assert abs(int(b[0]) - math.ceil(tau * N)) <= 20
+    assert 1 <= b[1] < 100                                     # a sharp row keeps a handful of keys
+    sig = np.sqrt(2 * np.maximum(0.0, math.log(N) - H.astype(np.float64)))
+    ref = np.ceil(N * scipy.stats.norm.sf(sig - scipy.stats.norm.ppf(tau)))
+    assert np.array_equal(b, np.clip(ref, 1, N).astype(np.int32))
+    # the defining property: the largest B*N of N lognormal weights hold mass tau
+    for s_, B in zip(sig[2:5], (N * scipy.stats.norm.sf(sig - scipy.stats.norm.ppf(tau)))[2:5] / N):
+        assert abs(scipy.stats.norm.sf(scipy.stats.norm.ppf(1 - B) - s_) - tau) < 1e-9
+    hs = np.linspace(0, math.log(N), 3000).astype(np.float32)
+    bs, _ = oracle.budget_lognormal(hs, tau, N)
+    assert np.all(np.diff(bs) >= 0)                            # monotone in entropy
+    # Table of the appendix: the lognormal map over-estimates relative to the uniform one at
+    # mid entropies (mean error +0.0164 vs -0.0415) -- its budgets are the larger ones there
+    bu, _ = oracle.budget(hs, tau, N)
+    mid = (hs > 0.5 * math.log(N)) & (hs < 0.95 * math.log(N))
+    assert np.all(bs[mid] >= bu[mid])
+
+
 # ----------------------------------------------------------------------------- grid count
 def gauss_circle():
     with open(os.path.join(GOLDEN, "gauss_circle.txt")) as f:
