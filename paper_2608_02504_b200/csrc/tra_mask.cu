@@ -25,7 +25,8 @@
 //    c(y', x') = #{queries i : (x'-x_i)^2 + (y'-y_i)^2 <= theta[ridx_i][|f - t_i|]} is built for
 //    the whole frame at once: a query's disk meets row y' in the x-interval of half-width
 //    floor(sqrt(theta - (y'-y_i)^2)), which adds +1 / -1 to a difference array in shared
-//    memory; a prefix sum along each row turns it into the counts.  Every undecided key block
+//    memory; a prefix sum along each row turns it into the counts (a disk that covers the whole
+//    frame is only counted once, a disk that covers a whole row skips the square root).  Every undecided key block
 //    then reads the counts of its own keys in that frame (c_j by definition) and accumulates
 //    its numbers of reached and of high columns.
 // The outcome equals the unpruned vote bit for bit.
@@ -46,9 +47,9 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   extern __shared__ int32_t s_dyn[];
   __shared__ int s_rank_ridx[128];
   __shared__ tra_block_boxes_t s_ubox;
-  __shared__ int s_rstar, s_count;
+  __shared__ int s_rstar, s_count, s_whole;
 
-  const int Wp = W + 1;
+  const int Wp = (W + 1) | 1;                                      // odd row stride
   int32_t* s_theta_star = s_dyn;                                   // [T]
   int32_t* s_frame_needed = s_dyn + T;                             // [T]
   int32_t* s_diff = s_dyn + 2 * T;                                 // [H * (W + 1)]
@@ -145,37 +146,50 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   for (int f = 0; f < T; ++f) {
     if (!s_frame_needed[f]) continue;                   // uniform across the CTA
     for (int i = tid; i < H * Wp; i += TRA_MASK_THREADS) s_diff[i] = 0;
+    if (tid == 0) s_whole = 0;
     __syncthreads();
     if (tid < nq) {
       const int th = __ldg(theta + qr * T + abs(qt - f));
-      const int R = tra_isqrt_small(th);
-      const int ylo = max(0, qy - R), yhi = min(H - 1, qy + R);
-      for (int yy = ylo; yy <= yhi; ++yy) {
-        const int dy = yy - qy;
-        const int w = tra_isqrt_small(th - dy * dy);
-        atomicAdd(&s_diff[yy * Wp + max(0, qx - w)], 1);
-        atomicAdd(&s_diff[yy * Wp + min(W - 1, qx + w) + 1], -1);
+      const int far_x = max(qx, W - 1 - qx), far_y = max(qy, H - 1 - qy);
+      if (th >= far_x * far_x + far_y * far_y) {
+        atomicAdd(&s_whole, 1);                       // the disk covers the whole frame
+      } else {
+        const int R = tra_isqrt_small(th);
+        const int ylo = max(0, qy - R), yhi = min(H - 1, qy + R);
+        for (int yy = ylo; yy <= yhi; ++yy) {
+          const int dy = yy - qy;
+          const int rem = th - dy * dy;
+          int lo = 0, hi = W;                         // the disk covers the whole row ...
+          if (rem < far_x * far_x) {                  // ... unless its half-width falls short
+            const int w = tra_isqrt_small(rem);
+            lo = max(0, qx - w);
+            hi = min(W - 1, qx + w) + 1;
+          }
+          atomicAdd(&s_diff[yy * Wp + lo], 1);
+          atomicAdd(&s_diff[yy * Wp + hi], -1);
+        }
       }
     }
     __syncthreads();
-    // prefix sum along x, one warp per row
-    for (int yy = warp; yy < H; yy += TRA_MASK_WARPS) {
-      int carry = 0;
-      for (int x0 = 0; x0 < W; x0 += 32) {
-        const int x = x0 + lane;
-        int val = x < W ? s_diff[yy * Wp + x] : 0;
+    // prefix sum along x: one thread per row (the row stride W + 1 is made odd, so the threads
+    // of a warp walk different banks)
+    for (int yy = tid; yy < H; yy += TRA_MASK_THREADS) {
+      int32_t* row = s_diff + yy * Wp;
+      int run = 0;
+      for (int x0 = 0; x0 < W; x0 += 8) {          // eight independent loads, then the running sum
+        int v[8];
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-          int other = __shfl_up_sync(0xffffffffu, val, off);
-          if (lane >= off) val += other;
+        for (int j = 0; j < 8; ++j) v[j] = x0 + j < W ? row[x0 + j] : 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          run += v[j];
+          if (x0 + j < W) row[x0 + j] = run;
         }
-        val += carry;
-        if (x < W) s_diff[yy * Wp + x] = val;
-        carry = __shfl_sync(0xffffffffu, val, 31);
       }
     }
     __syncthreads();
     // undecided key blocks with tokens in this frame: one warp per block
+    const int whole = s_whole;                         // queries whose disk covers every key of the frame
     const int p_begin = f * HW, p_end = min(N, (f + 1) * HW);
     const int v_first = p_begin / b, v_last = (p_end - 1) / b;
     for (int v = v_first + warp; v <= v_last; v += TRA_MASK_WARPS) {
@@ -187,7 +201,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
         int c = 0;
         if (p < pe) {
           const uint32_t kc = coord_packed[p];
-          c = s_diff[tra_coord_y(kc) * Wp + tra_coord_x(kc)];
+          c = s_diff[tra_coord_y(kc) * Wp + tra_coord_x(kc)] + whole;
         }
         ne += __popc(__ballot_sync(0xffffffffu, c > 0));
         hi += __popc(__ballot_sync(0xffffffffu, 3 * c > b));
@@ -283,7 +297,7 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   const long long rows = BH * NB;
 
   const int H = plan->cfg.H, W = plan->cfg.W;
-  size_t smem = ((size_t)2 * T + (size_t)H * (W + 1)) * sizeof(int32_t) + (size_t)NB * 5;
+  size_t smem = ((size_t)2 * T + (size_t)H * ((W + 1) | 1)) * sizeof(int32_t) + (size_t)NB * 5;
   smem = (smem + 15) & ~(size_t)15;
   if (smem > 200 * 1024) return TRA_ERR_UNSUPPORTED;     // frame too large for the count field
   dim3 grid((unsigned)NB, (unsigned)BH);
