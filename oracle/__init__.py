@@ -153,20 +153,22 @@ def token_mask_row(coord, T, theta, qi, ridx_q):
     return row.astype(bool)
 
 
-def block_vote(coord, T, b, theta, ridx_head, u_list=None, keep_diagonal=False):
-    """Algorithm 1 for one head: uint8 [len(u_list), NB], no bounding-box shortcut."""
+def block_vote(coord, T, b, theta, ridx_head, u_list=None, keep_diagonal=False, n_text=0):
+    """Algorithm 1 for one head: uint8 [len(u_list), NB], no bounding-box shortcut.
+    n_text text tokens follow the video tokens; their blocks stay dense."""
     coord = _c(coord, np.int32)
     theta = _c(theta, np.int32)
     ridx_head = _c(ridx_head, np.uint16)
     N = coord.shape[0]
-    NB = (N + b - 1) // b
+    NB = (N + n_text + b - 1) // b
     if u_list is None:
         u_list = np.arange(NB)
     u_list = _c(u_list, np.int32)
     out = np.empty((u_list.size, NB), np.uint8)
     lib().tra_oracle_block_vote(_ptr(coord, ctypes.c_int32), N, T, b, _ptr(theta, ctypes.c_int32),
                                 _ptr(ridx_head, ctypes.c_uint16), _ptr(u_list, ctypes.c_int32),
-                                u_list.size, int(bool(keep_diagonal)), _ptr(out, ctypes.c_uint8))
+                                u_list.size, int(bool(keep_diagonal)), int(n_text),
+                                _ptr(out, ctypes.c_uint8))
     return out
 
 
@@ -180,19 +182,19 @@ def csr_from_block_mask(mask):
     return row_ptr, col_idx
 
 
-def visible_rows(coord, T, b, theta, ridx_head, rows, block_rows, mode):
-    """Visible key sets (bool [len(rows), N]) of the sparse pass; see the C source for modes."""
+def visible_rows(coord, T, b, theta, ridx_head, rows, block_rows, mode, n_text=0):
+    """Visible key sets (bool [len(rows), N + n_text]) of the sparse pass; see the C source for modes."""
     coord = _c(coord, np.int32)
     theta = _c(theta, np.int32)
     ridx_head = _c(ridx_head, np.uint16)
     rows = _c(rows, np.int32)
     N = coord.shape[0]
     block_rows = _c(block_rows, np.uint8) if block_rows is not None else None
-    vis = np.empty((rows.size, N), np.uint8)
+    vis = np.empty((rows.size, N + n_text), np.uint8)
     lib().tra_oracle_visible_rows(_ptr(coord, ctypes.c_int32), N, T, b,
                                   _ptr(theta, ctypes.c_int32), _ptr(ridx_head, ctypes.c_uint16),
                                   _ptr(rows, ctypes.c_int32), rows.size,
-                                  _ptr(block_rows, ctypes.c_uint8), mode,
+                                  _ptr(block_rows, ctypes.c_uint8), mode, int(n_text),
                                   _ptr(vis, ctypes.c_uint8))
     return vis
 

@@ -271,12 +271,22 @@ void tra_oracle_token_mask_row(const int32_t* coord, int N, int T, const int32_t
  * ------------------------------------------------------------------------- */
 void tra_oracle_block_vote(const int32_t* coord, int N, int T, int b, const int32_t* theta,
                            const uint16_t* ridx_head, const int32_t* u_list, int n_u,
-                           int keep_diagonal, uint8_t* out) {
-  int NB = (N + b - 1) / b;
+                           int keep_diagonal, int n_text, uint8_t* out) {
+  /* Joint text-video attention (Section 3.2, last paragraph; Algorithm 1): the sequence holds the
+   * N video tokens followed by n_text text tokens, S = N + n_text, NB = ceil(S / b) blocks of which
+   * the first B_v = ceil(N / b) are video blocks.  A pair with u >= B_v or v >= B_v is kept
+   * ("text or non-video blocks remain dense"); video blocks vote over their video tokens only
+   * (q < N, k < N), which is also what happens to the block that straddles the boundary. */
+  int NB = (N + n_text + b - 1) / b;
+  int NBv = (N + b - 1) / b;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int iu = 0; iu < n_u; ++iu) {
     int u = u_list[iu];
     for (int v = 0; v < NB; ++v) {
+      if (u >= NBv || v >= NBv) {
+        out[(size_t)iu * NB + v] = 1;
+        continue;
+      }
       int n_nonempty = 0, n_high = 0;
       for (int j = 0; j < b; ++j) {
         int k = v * b + j;
@@ -427,14 +437,19 @@ void tra_oracle_attention_rows_alg2(const uint16_t* Q, const uint16_t* K, const 
  * ------------------------------------------------------------------------- */
 void tra_oracle_visible_rows(const int32_t* coord, int N, int T, int b, const int32_t* theta,
                              const uint16_t* ridx_head, const int32_t* rows, int n_rows,
-                             const uint8_t* block_rows, int mode, uint8_t* visible) {
-  int NB = (N + b - 1) / b;
+                             const uint8_t* block_rows, int mode, int n_text, uint8_t* visible) {
+  /* With text tokens (positions N .. N + n_text - 1) the token mask applies to the video-key
+   * submatrix only: a text key, and any key seen from a text query, counts as inside the disk. */
+  int S = N + n_text;
+  int NB = (S + b - 1) / b;
   for (int r = 0; r < n_rows; ++r) {
     int qi = rows[r];
-    for (int j = 0; j < N; ++j) {
+    for (int j = 0; j < S; ++j) {
       int in_block = mode == 2 ? 1 : block_rows[(size_t)r * NB + j / b];
-      int in_disk = mode == 0 ? 1 : token_visible(coord, qi, j, theta, T, ridx_head[qi]);
-      visible[(size_t)r * N + j] = (uint8_t)(in_block && in_disk);
+      int in_disk = (mode == 0 || qi >= N || j >= N)
+                        ? 1
+                        : token_visible(coord, qi, j, theta, T, ridx_head[qi]);
+      visible[(size_t)r * S + j] = (uint8_t)(in_block && in_disk);
     }
   }
 }

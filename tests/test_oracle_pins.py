@@ -447,6 +447,37 @@ def test_ragged_last_block_rows_and_columns_do_not_exist():
     assert np.array_equal(out[0], numpy_block_vote(M, 32)[6])
 
 
+def test_text_tokens_keep_their_blocks_dense():
+    # Section 3.2 (last paragraph) and Algorithm 1: blocks with u >= B_v or v >= B_v are kept;
+    # video blocks vote over video tokens only; the token mask covers the video-key submatrix.
+    g = oracle.geometry(3, 7, 10, 4, 4, 32, 0.6, 0.9)          # N = 210: B_v = 7, block 6 straddles
+    n_text, b = 50, 32
+    S = g.N + n_text
+    NB = (S + b - 1) // b
+    assert NB == 9
+    rng = np.random.default_rng(8)
+    ridx = rng.integers(0, 8, S).astype(np.uint16)
+    with_text = oracle.block_vote(g.coord, g.T, b, g.theta, ridx, u_list=np.arange(NB), n_text=n_text)
+    video_only = oracle.block_vote(g.coord, g.T, b, g.theta, ridx[: g.N])
+    assert with_text.shape == (NB, NB)
+    assert np.array_equal(with_text[:7, :7], video_only)       # the video part is the video-only vote
+    assert with_text[7:, :].all() and with_text[:, 7:].all()   # text rows and text columns are dense
+    assert 0 < video_only.mean() < 1
+    rows = np.array([0, 100, 209, 210, 259])
+    M = numpy_token_mask(g, ridx[: g.N])
+    for mode in (0, 1, 2):
+        vis = oracle.visible_rows(g.coord, g.T, b, g.theta, ridx, rows, with_text[rows // b], mode,
+                                  n_text=n_text).astype(bool)
+        assert vis.shape == (rows.size, S)
+        blk = np.repeat(with_text[rows // b], b, axis=1)[:, :S].astype(bool)
+        tok = np.ones((rows.size, S), bool)
+        tok[:3, : g.N] = M[rows[:3]]                            # video queries: disks on video keys only
+        ref = {0: blk, 1: blk & tok, 2: tok}[mode]
+        assert np.array_equal(vis, ref)
+        assert vis[3:].all() if mode == 2 else True              # text queries see every key (Eq. 16 on video only)
+        assert vis[:, g.N:][:, :].all() if mode == 2 else True   # every text key is visible
+
+
 # ----------------------------------------------------------------------------- schedule
 def test_schedule_warmup_rule():
     with open(os.path.join(GOLDEN, "paper_schedule.txt")) as f:
