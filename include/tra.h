@@ -16,6 +16,13 @@
  * NB = ceil(N / block).  tra_tile_major_gather / _scatter move tensors between
  * raster order (n = (t*H + y)*W + x) and tile-major order.
  *
+ * Joint text-video attention (Section 3.2, last paragraph; Algorithm 1).  With cfg.n_text > 0 a
+ * sequence is the N video tokens followed by n_text text tokens, S = N + n_text; S takes the place
+ * of N in every shape below and NB = ceil(S / block).  The first B_v = ceil(N / block) blocks are
+ * video blocks; a block pair with u >= B_v or v >= B_v is always kept, video blocks vote over their
+ * video tokens only, the gather/scatter leaves text tokens where they are, and text positions get
+ * budget S, radius +inf and the last candidate index.
+ *
  * Shapes.  Q, K, V, O: bf16 [B, heads, N, head_dim].  entropy, budget, radius,
  * ridx: [B, heads, N].  block_mask: uint8 [B, heads, NB, NB].  row_ptr: int32
  * [B*heads*NB + 1]; col_idx: int32 [nnz], key blocks ascending inside a row.
@@ -66,6 +73,7 @@ typedef struct {
   int radius_policy;   /* TRA_RADII_* (used when radii == NULL)                                  */
   unsigned flags;      /* TRA_KEEP_DIAGONAL                                                      */
   int budget_map;      /* TRA_BUDGET_* used by tra_budget_radius                                 */
+  int n_text;          /* text tokens that follow the video tokens in every sequence (>= 0)     */
 } tra_config_t;
 
 /* ---- plan ---------------------------------------------------------------------------- */
@@ -80,7 +88,8 @@ int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* stream);
 int tra_plan_destroy(tra_plan_t* plan);
 
 /* Geometry queries (host). */
-int tra_plan_num_tokens(const tra_plan_t* plan);   /* N  */
+int tra_plan_num_tokens(const tra_plan_t* plan);   /* S = N + n_text: tokens per sequence */
+int tra_plan_num_video_tokens(const tra_plan_t* plan); /* N = T*H*W */
 int tra_plan_num_blocks(const tra_plan_t* plan);   /* NB */
 int tra_plan_num_radii(const tra_plan_t* plan);    /* |R| */
 /* Copies plan tables to HOST buffers (synchronises): radii[|R|] (double), theta[|R|*T]

@@ -23,7 +23,7 @@ TRA_BUDGET_UNIFORM = 0
 TRA_BUDGET_LOGNORMAL = 1
 
 EXPORTS = [
-    "tra_plan_create", "tra_plan_destroy", "tra_plan_num_tokens", "tra_plan_num_blocks",
+    "tra_plan_create", "tra_plan_destroy", "tra_plan_num_tokens", "tra_plan_num_video_tokens", "tra_plan_num_blocks",
     "tra_plan_num_radii", "tra_plan_tables", "tra_plan_count_table", "tra_plan_status",
     "tra_status_string", "tra_tile_major_gather", "tra_tile_major_scatter",
     "tra_entropy_attn", "tra_budget_radius", "tra_build_block_mask", "tra_sparse_attn",
@@ -38,6 +38,7 @@ class tra_config_t(ctypes.Structure):
         ("tau", ctypes.c_double), ("gamma", ctypes.c_double),
         ("radii", ctypes.POINTER(ctypes.c_double)), ("n_radii", ctypes.c_int),
         ("radius_policy", ctypes.c_int), ("flags", ctypes.c_uint), ("budget_map", ctypes.c_int),
+        ("n_text", ctypes.c_int),
     ]
 
 
@@ -50,7 +51,7 @@ def _load():
     vp, i32, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
     lib.tra_plan_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(tra_config_t), vp]
     lib.tra_plan_destroy.argtypes = [vp]
-    for name in ("tra_plan_num_tokens", "tra_plan_num_blocks", "tra_plan_num_radii"):
+    for name in ("tra_plan_num_tokens", "tra_plan_num_video_tokens", "tra_plan_num_blocks", "tra_plan_num_radii"):
         getattr(lib, name).argtypes = [vp]
     lib.tra_plan_tables.argtypes = [vp, vp, vp, vp]
     lib.tra_plan_count_table.argtypes = [vp, vp]
@@ -97,7 +98,8 @@ class Plan:
     """Owns a ``tra_plan_t`` (geometry, thresholds, count table, block boxes)."""
 
     def __init__(self, T, H, W, head_dim, block, tile_h, tile_w, tau=0.9, gamma=0.6, radii=None,
-                 radius_policy=TRA_RADII_EXTENDED, flags=0, budget_map=TRA_BUDGET_UNIFORM, stream=None):
+                 radius_policy=TRA_RADII_EXTENDED, flags=0, budget_map=TRA_BUDGET_UNIFORM, n_text=0,
+                 stream=None):
         cfg = tra_config_t()
         cfg.T, cfg.H, cfg.W = T, H, W
         cfg.head_dim, cfg.block, cfg.tile_h, cfg.tile_w = head_dim, block, tile_h, tile_w
@@ -109,10 +111,12 @@ class Plan:
             cfg.radii = ctypes.cast(arr, ctypes.POINTER(ctypes.c_double))
             cfg.n_radii = len(radii)
         cfg.radius_policy, cfg.flags, cfg.budget_map = radius_policy, flags, budget_map
+        cfg.n_text = n_text
         self.cfg = cfg
         self._h = ctypes.c_void_p()
         _check(_lib.tra_plan_create(ctypes.byref(self._h), ctypes.byref(cfg), _stream(stream)), "tra_plan_create")
-        self.N = _lib.tra_plan_num_tokens(self._h)
+        self.N = _lib.tra_plan_num_tokens(self._h)              # tokens per sequence (video + text)
+        self.N_video = _lib.tra_plan_num_video_tokens(self._h)
         self.NB = _lib.tra_plan_num_blocks(self._h)
         self.n_radii = _lib.tra_plan_num_radii(self._h)
         self.T, self.H, self.W = T, H, W
@@ -141,7 +145,7 @@ class Plan:
         import numpy as np
         radii = np.empty(self.n_radii, np.float64)
         theta = np.empty((self.n_radii, self.T), np.int32)
-        coord = np.empty((self.N, 3), np.int32)
+        coord = np.empty((self.N_video, 3), np.int32)
         _check(_lib.tra_plan_tables(self._h, radii.ctypes.data, theta.ctypes.data, coord.ctypes.data),
                "tra_plan_tables")
         return radii, theta, coord

@@ -770,15 +770,15 @@ int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, 
   using C = Cfg<D, BN>;
   CUtensorMap mq, mk, mv;
   int rc;
-  if ((rc = make_map(&mq, Q, D, plan->N, BH, kTileM)) != TRA_OK) return rc;
-  if ((rc = make_map(&mk, K, D, plan->N, BH, BN)) != TRA_OK) return rc;
-  if ((rc = make_map(&mv, V, D, plan->N, BH, BN)) != TRA_OK) return rc;
+  if ((rc = make_map(&mq, Q, D, plan->S, BH, kTileM)) != TRA_OK) return rc;
+  if ((rc = make_map(&mk, K, D, plan->S, BH, BN)) != TRA_OK) return rc;
+  if ((rc = make_map(&mv, V, D, plan->S, BH, BN)) != TRA_OK) return rc;
   auto kern = tra_attn_kernel<D, BN, kEntropy>;
   TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-  const int n_pairs = (plan->N + 2 * kTileM - 1) / (2 * kTileM);
+  const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
   dim3 grid((unsigned)n_pairs, (unsigned)BH);
   kern<<<grid, kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, (__nv_bfloat16*)O, entropy, lse, row_ptr,
-                                                  col_idx, plan->N, plan->NB, sm_scale * kLog2e,
+                                                  col_idx, plan->S, plan->NB, sm_scale * kLog2e,
                                                   plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;

@@ -24,7 +24,8 @@ static_assert(sizeof(tra_block_boxes_t) == 80, "block boxes");
 
 struct tra_plan {
   tra_config_t cfg;
-  int N, NB, n_radii;
+  int N, NB, n_radii;   // N = T*H*W video tokens; NB = blocks of the whole sequence
+  int S, NBv;           // S = N + n_text tokens in the sequence; NBv = ceil(N / block) video blocks
   int device;
   double z_tau;       // Phi^-1(tau), for the lognormal budget map
   // host copies

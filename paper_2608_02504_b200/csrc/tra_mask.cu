@@ -42,8 +42,8 @@ __device__ __forceinline__ int tra_isqrt_small(int n) {
 __global__ void __launch_bounds__(TRA_MASK_THREADS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
-                      uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int NB,
-                      int b, int T, int H, int W, int keep_diagonal) {
+                      uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int S, int NB,
+                      int NBv, int b, int T, int H, int W, int keep_diagonal) {
   extern __shared__ int32_t s_dyn[];
   __shared__ int s_rank_ridx[128];
   __shared__ tra_block_boxes_t s_ubox;
@@ -60,9 +60,15 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x;
   const long long bh = blockIdx.y;
-  const uint16_t* ridx_h = ridx + bh * N;
+  const uint16_t* ridx_h = ridx + bh * S;
   uint8_t* mask_row = block_mask + (bh * NB + u) * (long long)NB;
 
+  // Text rows (u >= NBv) keep every block (Algorithm 1: "text or non-video blocks remain dense").
+  if (u >= NBv) {
+    for (int v = tid; v < NB; v += TRA_MASK_THREADS) mask_row[v] = 1;
+    if (tid == 0) row_ptr[bh * NB + u + 1] = NB;
+    return;
+  }
   const int q0 = u * b;
   const int nq = min(b, N - q0);                       // valid queries of this block
   const int need = b / 3 + 1;
@@ -109,7 +115,9 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   int kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
     int decided = 0;   // 0 = vote 0, 1 = vote 1, 2 = undecided
-    if (rstar >= 0) {
+    if (v >= NBv) {
+      decided = 1;     // text key block
+    } else if (rstar >= 0) {
       tra_block_boxes_t vb = boxes[v];
       bool all_reject = true, all_accept = true;
       for (int iu = 0; iu < s_ubox.n_box; ++iu) {
@@ -191,7 +199,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     // undecided key blocks with tokens in this frame: one warp per block
     const int whole = s_whole;                         // queries whose disk covers every key of the frame
     const int p_begin = f * HW, p_end = min(N, (f + 1) * HW);
-    const int v_first = p_begin / b, v_last = (p_end - 1) / b;
+    const int v_first = p_begin / b, v_last = (p_end - 1) / b;     // video blocks only: p_end <= N
     for (int v = v_first + warp; v <= v_last; v += TRA_MASK_WARPS) {
       if (s_state[v] != 2) continue;
       const int ps = max(v * b, p_begin), pe = min((v + 1) * b, p_end);
@@ -305,7 +313,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_block_vote_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)smem));
   tra_block_vote_kernel<<<grid, TRA_MASK_THREADS, smem, stream>>>(
-      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, NB,
+      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, plan->S, NB,
+      plan->NBv,
       plan->cfg.block, T, H, W, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,

@@ -61,14 +61,14 @@ __global__ void tra_count_table_kernel(int T, int H, int W, int n_radii,
 template <bool kGather>
 __global__ void tra_permute_rows_kernel(const int32_t* __restrict__ raster_of_pos,
                                         const uint4* __restrict__ src, uint4* __restrict__ dst,
-                                        int N, int chunks_per_row, long long total_chunks) {
+                                        int N, int S, int chunks_per_row, long long total_chunks) {
   long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= total_chunks) return;
   int chunk = (int)(g % chunks_per_row);
-  long long row = g / chunks_per_row;  // bh * N + p
-  int p = (int)(row % N);
-  long long bh = row / N;
-  long long other = bh * N + raster_of_pos[p];
+  long long row = g / chunks_per_row;  // bh * S + p
+  int p = (int)(row % S);
+  long long bh = row / S;
+  long long other = bh * S + (p < N ? raster_of_pos[p] : p);   // text tokens stay in place
   if (kGather)
     dst[row * chunks_per_row + chunk] = src[other * chunks_per_row + chunk];
   else
@@ -118,13 +118,16 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   if ((long long)T * H * W > (1ll << 30)) return TRA_ERR_UNSUPPORTED;
   if (cfg->budget_map != TRA_BUDGET_UNIFORM && cfg->budget_map != TRA_BUDGET_LOGNORMAL)
     return TRA_ERR_INVALID_ARG;
+  if (cfg->n_text < 0 || cfg->n_text > (1 << 24)) return TRA_ERR_INVALID_ARG;
 
   tra_plan* p = new tra_plan();
   memset(p, 0, sizeof(*p));
   p->cfg = *cfg;
   p->cfg.radii = nullptr;
   p->N = T * H * W;
-  p->NB = (p->N + cfg->block - 1) / cfg->block;
+  p->S = p->N + cfg->n_text;
+  p->NB = (p->S + cfg->block - 1) / cfg->block;
+  p->NBv = (p->N + cfg->block - 1) / cfg->block;
   p->z_tau = tra_inverse_normal_cdf(cfg->tau);
   if (cudaGetDevice(&p->device) != cudaSuccess) {
     delete p;
@@ -215,7 +218,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
         }
   }
   std::vector<tra_block_boxes_t> boxes(p->NB);
-  for (int u = 0; u < p->NB; ++u) {
+  for (int u = 0; u < p->NB; ++u) {   // text-only blocks keep n_box = 0
     tra_block_boxes_t bb;
     memset(&bb, 0, sizeof(bb));
     int nb = 0, last_tile = -1;
@@ -280,7 +283,8 @@ extern "C" int tra_plan_destroy(tra_plan_t* plan) {
   return TRA_OK;
 }
 
-extern "C" int tra_plan_num_tokens(const tra_plan_t* plan) { return plan ? plan->N : TRA_ERR_INVALID_ARG; }
+extern "C" int tra_plan_num_tokens(const tra_plan_t* plan) { return plan ? plan->S : TRA_ERR_INVALID_ARG; }
+extern "C" int tra_plan_num_video_tokens(const tra_plan_t* plan) { return plan ? plan->N : TRA_ERR_INVALID_ARG; }
 extern "C" int tra_plan_num_blocks(const tra_plan_t* plan) { return plan ? plan->NB : TRA_ERR_INVALID_ARG; }
 extern "C" int tra_plan_num_radii(const tra_plan_t* plan) { return plan ? plan->n_radii : TRA_ERR_INVALID_ARG; }
 
@@ -327,15 +331,15 @@ static int tra_permute(const tra_plan_t* plan, const void* src, void* dst, int n
   if (((uintptr_t)src & 15) || ((uintptr_t)dst & 15)) return TRA_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)stream_;
   int chunks = row_bytes / 16;
-  long long total = (long long)n_bh * plan->N * chunks;
+  long long total = (long long)n_bh * plan->S * chunks;
   long long grid = (total + 255) / 256;
   if (grid > 0x7fffffffll) return TRA_ERR_UNSUPPORTED;
   if (gather)
     tra_permute_rows_kernel<true><<<(unsigned)grid, 256, 0, stream>>>(
-        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, chunks, total);
+        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, plan->S, chunks, total);
   else
     tra_permute_rows_kernel<false><<<(unsigned)grid, 256, 0, stream>>>(
-        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, chunks, total);
+        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, plan->S, chunks, total);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }

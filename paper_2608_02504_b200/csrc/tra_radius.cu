@@ -13,11 +13,17 @@ __global__ void tra_budget_radius_kernel(const float* __restrict__ entropy,
                                          const uint32_t* __restrict__ counts,
                                          const float* __restrict__ radii, int32_t* __restrict__ budget,
                                          float* __restrict__ radius, uint16_t* __restrict__ ridx,
-                                         int N, int H, int W, int n_radii, double tau,
+                                         int N, int S, int H, int W, int n_radii, double tau,
                                          int budget_map, double z_tau, double log_n, long long total) {
   long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= total) return;
-  int p = (int)(g % N);
+  int p = (int)(g % S);
+  if (p >= N) {                      // text token: sees every key (Section 3.2, last paragraph)
+    if (budget) budget[g] = S;
+    if (radius) radius[g] = INFINITY;
+    ridx[g] = (uint16_t)(n_radii - 1);
+    return;
+  }
   double v;
   if (budget_map == TRA_BUDGET_LOGNORMAL) {
     // sigma = sqrt(2 (log N - H)),  B = Phibar(sigma - Phi^-1(tau)),  K = ceil(N B)
@@ -47,12 +53,12 @@ extern "C" int tra_budget_radius(const tra_plan_t* plan, const float* entropy, i
                                  float* radius, uint16_t* ridx, int B, int heads, void* stream_) {
   if (!plan || !entropy || !ridx || B < 1 || heads < 1) return TRA_ERR_INVALID_ARG;
   cudaStream_t stream = (cudaStream_t)stream_;
-  long long total = (long long)B * heads * plan->N;
+  long long total = (long long)B * heads * plan->S;
   long long grid = (total + 255) / 256;
   if (grid > 0x7fffffffll) return TRA_ERR_UNSUPPORTED;
   tra_budget_radius_kernel<<<(unsigned)grid, 256, 0, stream>>>(
       entropy, plan->d_coord_packed, plan->d_counts, plan->d_radii_f32, budget, radius, ridx,
-      plan->N, plan->cfg.H, plan->cfg.W, plan->n_radii, plan->cfg.tau, plan->cfg.budget_map, plan->z_tau,
+      plan->N, plan->S, plan->cfg.H, plan->cfg.W, plan->n_radii, plan->cfg.tau, plan->cfg.budget_map, plan->z_tau,
       log((double)plan->N), total);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;

@@ -94,6 +94,29 @@ def make_qkv(cfg, device="cpu", heads=None):
     return Q, K, V
 
 
+def append_text(Q, K, V, cfg, n_text: int, heads=None):
+    """Joint text-video sequences: n_text text tokens after the video tokens of every head.
+    Text tokens carry no position embedding: q = s * u, k = u', v ~ N(0, 1), from a generator of
+    their own, so the video part is the tensor make_qkv returns.  Returns new [1, heads, N + n_text, d]."""
+    heads = list(range(cfg["heads"])) if heads is None else list(heads)
+    d, device = cfg["head_dim"], Q.device
+    out = [torch.empty(1, len(heads), Q.shape[2] + n_text, d, dtype=torch.bfloat16, device=device) for _ in range(3)]
+    for src, dst in zip((Q, K, V), out):
+        dst[:, :, : Q.shape[2]] = src
+    for i, h in enumerate(heads):
+        g = torch.Generator(device=device)
+        g.manual_seed(cfg["seed"] * 1000003 + 500000 + h)
+        u = torch.randn(n_text, d, generator=g, device=device)
+        u2 = torch.randn(n_text, d, generator=g, device=device)
+        v = torch.randn(n_text, d, generator=g, device=device)
+        r = torch.rand(n_text, generator=g, device=device)
+        s = torch.exp(math.log(cfg["s_lo"]) + r * (math.log(cfg["s_hi"]) - math.log(cfg["s_lo"])))
+        out[0][0, i, Q.shape[2]:] = (s[:, None] * u).to(torch.bfloat16)
+        out[1][0, i, Q.shape[2]:] = u2.to(torch.bfloat16)
+        out[2][0, i, Q.shape[2]:] = v.to(torch.bfloat16)
+    return tuple(out)
+
+
 def drift_(x: torch.Tensor, step: int, seed: int, sigma: float = 0.05) -> torch.Tensor:
     """Denoising-schedule emulation: x_t = x_{t-1} + sigma * N(0, 1), in place on an fp32 state."""
     g = torch.Generator(device=x.device)

@@ -395,6 +395,60 @@ def test_full_size_sampled_rows(name, heads_checked, n_random):
     plan.close()
 
 
+# ----------------------------------------------------------------------------- joint text-video attention
+TEXT_CASES = [(CFG_TINY, 40), (CFG_RAGGED64, 50), (CFG_RAGGED128, 200), (CFG_MID128, 100)]
+
+
+@pytest.mark.parametrize("cfg,n_text", TEXT_CASES, ids=["tiny+40", "ragged64+50", "ragged128+200", "mid128+100"])
+def test_text_tokens_pipeline(cfg, n_text):
+    """Section 3.2 (last paragraph) / Algorithm 1 with S = N + n_text: text tokens stay in place in
+    the tile-major order, get the full-support candidate, their blocks are dense, video blocks vote
+    over video tokens only, and both attentions run over the whole sequence."""
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg, n_text=n_text)
+    S, b = geo.N + n_text, geo.block
+    NB = (S + b - 1) // b
+    assert plan.N == S and plan.N_video == geo.N and plan.NB == NB
+    Qr, Kr, Vr = workloads.append_text(*workloads.make_qkv(cfg, DEV), cfg, n_text)
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    perm = np.concatenate([common.raster_of_pos(geo), np.arange(geo.N, S)])
+    assert torch.equal(Q.cpu(), Qr.cpu()[:, :, torch.from_numpy(perm).long(), :])
+    assert torch.equal(plan.tile_major_scatter(Q), Qr)
+
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    budget, radius, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    plan.check_status()
+
+    Hn = H.cpu().numpy()[0]
+    ridx_np = ridx.cpu().numpy().view(np.uint16)[0]
+    assert np.all(ridx_np[:, geo.N:] == geo.radii.size - 1)
+    assert np.all(budget.cpu().numpy()[0][:, geo.N:] == S)
+    assert np.all(np.isinf(radius.cpu().numpy()[0][:, geo.N:]))
+    bud_ref, fragile = oracle.budget(Hn[:, : geo.N], geo.tau, geo.N)
+    assert not fragile.any()
+    ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)
+    assert np.array_equal(ridx_np[:, : geo.N], ridx_ref)
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(S)
+    for h in range(cfg["heads"]):
+        dense = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows)
+        common.assert_output(O[0, h], dense["O"], f"dense+text head {h}")
+        assert np.abs(Hn[h] - dense["H_def"]).max() <= common.ENTROPY_ATOL
+        ref_mask = oracle.block_vote(geo.coord, geo.T, b, geo.theta, ridx_np[h], u_list=np.arange(NB),
+                                     n_text=n_text)
+        assert np.array_equal(mask[0, h].cpu().numpy(), ref_mask)
+        vis = oracle.visible_rows(geo.coord, geo.T, b, geo.theta, ridx_np[h], rows, ref_mask[rows // b], 0,
+                                  n_text=n_text)
+        ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis)
+        common.assert_output(Os[0, h], ref["O"], f"sparse+text head {h}")
+    rp, ci = oracle.csr_from_block_mask(mask[0].cpu().numpy())
+    assert np.array_equal(row_ptr.cpu().numpy().astype(np.int64), rp)
+    assert np.array_equal(col_idx.cpu().numpy()[: int(nnz.item())], ci)
+    plan.close()
+
+
 # ----------------------------------------------------------------------------- reuse across steps
 def test_mask_reuse_across_denoising_steps():
     """Warm-up reuse (Section 3.3): radii and mask of the last dense step serve every later step;
