@@ -104,6 +104,12 @@ int tra_plan_status(tra_plan_t* plan, void* stream);
 
 const char* tra_status_string(int status);
 
+/* Self-test of the device-side error path (the paper has no counterpart): launches one warp that
+ * waits, with the same bounded wait the attention kernels use, on a barrier nothing arrives on.
+ * After limit_ms (1..1000) the wait gives up and records TRA_ERR_TIMEOUT in the plan status; the
+ * kernel then returns normally and the context stays usable.  Asynchronous on `stream`. */
+int tra_selftest_wait_timeout(tra_plan_t* plan, int limit_ms, void* stream);
+
 /* ---- layout (Section 3.3: Q, K, V are reordered before attention, O restored after) -- */
 
 /* dst[bh, p, :] = src[bh, raster(p), :] for every tile-major position p.  row_bytes = bytes of

@@ -25,7 +25,7 @@ TRA_BUDGET_LOGNORMAL = 1
 EXPORTS = [
     "tra_plan_create", "tra_plan_destroy", "tra_plan_num_tokens", "tra_plan_num_video_tokens", "tra_plan_num_blocks",
     "tra_plan_num_radii", "tra_plan_tables", "tra_plan_count_table", "tra_plan_status",
-    "tra_status_string", "tra_tile_major_gather", "tra_tile_major_scatter",
+    "tra_status_string", "tra_selftest_wait_timeout", "tra_tile_major_gather", "tra_tile_major_scatter",
     "tra_entropy_attn", "tra_budget_radius", "tra_build_block_mask", "tra_sparse_attn",
 ]
 
@@ -57,6 +57,7 @@ def _load():
     lib.tra_plan_count_table.argtypes = [vp, vp]
     lib.tra_plan_status.argtypes = [vp, vp]
     lib.tra_status_string.argtypes = [i32]
+    lib.tra_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.tra_status_string.restype = ctypes.c_char_p
     lib.tra_tile_major_gather.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.tra_tile_major_scatter.argtypes = [vp, vp, vp, i32, i32, vp]
@@ -158,6 +159,10 @@ class Plan:
 
     def status(self, stream=None):
         return _lib.tra_plan_status(self._h, _stream(stream))
+
+    def selftest_wait_timeout(self, limit_ms=20):
+        """Runs the bounded-wait self-test kernel; the plan status then reads TRA_ERR_TIMEOUT."""
+        _check(_lib.tra_selftest_wait_timeout(self._h, limit_ms, _stream()), "tra_selftest_wait_timeout")
 
     def check_status(self, stream=None):
         _check(self.status(stream), "tra_plan_status")

@@ -77,13 +77,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 }
 // Bounded wait; false = gave up (abort flag raised by this or another thread).
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            int* status) {
+                                            int* status, unsigned long long limit_ns = kWaitLimitNs) {
   const unsigned long long t0 = globaltimer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      if (globaltimer_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         tra_set_status(status, TRA_ERR_TIMEOUT);
         return false;
@@ -810,7 +810,28 @@ int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const vo
   return TRA_ERR_UNSUPPORTED;
 }
 
+// Self-test of the bounded wait: one warp waits on an mbarrier that nothing ever arrives on.
+__global__ void tra_wait_timeout_selftest_kernel(unsigned long long limit_ns, int* status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) mbar_wait_slow(smem_u32(&bar), 0u, &abort_flag, status, limit_ns);
+}
+
 }  // namespace
+
+extern "C" int tra_selftest_wait_timeout(tra_plan_t* plan, int limit_ms, void* stream) {
+  if (!plan || limit_ms < 1 || limit_ms > 1000) return TRA_ERR_INVALID_ARG;
+  tra_wait_timeout_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(
+      (unsigned long long)limit_ms * 1000000ull, plan->d_status);
+  TRA_CUDA_CHECK(cudaGetLastError());
+  return TRA_OK;
+}
 
 extern "C" int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
                                 void* O, float* entropy, float* lse, int B, int heads, float sm_scale,

@@ -484,6 +484,22 @@ def test_mask_reuse_across_denoising_steps():
     plan.close()
 
 
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A device-side wait that can never be satisfied gives up after its limit, records
+    TRA_ERR_TIMEOUT in the plan status and the kernel returns; later calls work normally."""
+    cfg = CFG_TINY
+    plan = make_plan(cfg)
+    assert plan.status() == 0
+    plan.selftest_wait_timeout(limit_ms=20)
+    assert plan.status() == -5          # TRA_ERR_TIMEOUT
+    assert plan.status() == 0           # cleared by the read
+    Q, K, V = tile_major_inputs(cfg, plan)
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    plan.check_status()
+    assert torch.isfinite(H).all() and torch.isfinite(O.float()).all()
+    plan.close()
+
+
 def test_attention_rejects_bad_arguments():
     a = api()
     plan = make_plan(CFG_TINY)
