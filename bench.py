@@ -9,8 +9,8 @@ One "step" is one pass of the whole hot path over one layer's synthetic Q/K/V at
 
 `value` is the effective throughput of the pass, 4*d*(computed query-key pairs)/time summed
 over the dense and the sparse attention of the step, with inputs resident in HBM.  The JSON
-line also carries per-stage times (`stages`), the sparse kernel's roofline (`roofline`), the
-dense kernel's (`roofline_dense`), the 50-step denoising-schedule emulation (`schedule`), the
+line also carries per-stage times (`stages`), the roofline of the dominant kernel (`roofline`:
+the fused dense + entropy launch) and of the sparse launch (`roofline_sparse`), the 50-step denoising-schedule emulation (`schedule`), the
 end-to-end number with host buffers (`e2e`) and the fp64 oracle timed on the host cores
 (`cpu_baseline`).
 
@@ -46,6 +46,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # the ncu capture of a 4-head case summarised in profiles/attention_kernels_wan14b-720p_4heads.md
 # (234.4 MB + 59.3 MB for 4 heads); traffic grows in proportion to the head count.
 NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (234.363648e6 + 59.300864e6) / 4
+NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (233.931520e6 + 63.376128e6) / 4
 
 
 def load_peaks():
@@ -298,16 +299,20 @@ def run_ours(args):
         "gather_gbs": round(3 * 2 * heads * N * row_bytes / (stage_ms["gather"]["mean"] * 1e-3) / 1e9, 1),
     }
 
-    roofline = {"bound": "tensor", "kernel": "tra_attn_kernel<128,128,false> (block-sparse attention)",
-                "achieved": round(tf_sparse, 2), "peak": peak_tf, "unit": "TFLOP/s",
-                "frac": round(tf_sparse / peak_tf, 4),
-                "traffic": (NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD * heads if args.config == "wan14b-720p" else None),
-                "peak_source": peak_note, "flops_per_launch": 4.0 * d * pairs_sparse,
-                "launch_ms": round(t_sparse * 1e3, 4)}
-    roofline_dense = {"bound": "tensor", "kernel": "tra_attn_kernel<128,128,true> (dense attention + entropy)",
-                      "achieved": round(tf_dense, 2), "peak": peak_tf, "unit": "TFLOP/s",
-                      "frac": round(tf_dense / peak_tf, 4), "traffic": None, "peak_source": peak_note,
-                      "flops_per_launch": 4.0 * d * pairs_dense, "launch_ms": round(t_dense * 1e3, 4)}
+    # `roofline` is the kernel that dominates the step (the fused dense + entropy launch, ~70 % of a
+    # pass); `roofline_sparse` is the same kernel family on the retained blocks (the sparse layer).
+    def attn_roofline(kernel, tflops, flops, seconds, traffic):
+        return {"bound": "tensor", "kernel": kernel, "achieved": round(tflops, 2), "peak": peak_tf,
+                "unit": "TFLOP/s", "frac": round(tflops / peak_tf, 4), "traffic": traffic,
+                "peak_source": peak_note, "flops_per_launch": flops, "launch_ms": round(seconds * 1e3, 4)}
+
+    full_shape = args.config == "wan14b-720p"
+    roofline = attn_roofline("tra_attn_kernel<128,128,true> (dense attention + entropy)", tf_dense,
+                             4.0 * d * pairs_dense, t_dense,
+                             NCU_DENSE_TRAFFIC_BYTES_PER_HEAD * heads if full_shape else None)
+    roofline_sparse = attn_roofline("tra_attn_kernel<128,128,false> (block-sparse attention)", tf_sparse,
+                                    4.0 * d * pairs_sparse, t_sparse,
+                                    NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD * heads if full_shape else None)
 
     # ---- target-mass sweep: the paper's 9-19 % density band is reached at smaller tau -----------
     tau_sweep = None
@@ -377,7 +382,7 @@ def run_ours(args):
                        "parallelism": f"replicated layer per GPU x{world} (heads/batch shard, no collective)",
                        "l2": "inputs larger than L2 (Q/K/V/O are 774 MB each)"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "roofline_dense": roofline_dense, "stages": stages,
+            "roofline": roofline, "roofline_sparse": roofline_sparse, "stages": stages,
             "tau_sweep": tau_sweep, "schedule": schedule, "cpu_baseline": cpu_baseline,
             "paper_context": "paper: 1.56-2.05x end-to-end speedup at 9-19% retained interactions on one H200",
             "wall_s_timed_region": round(wall_s, 3),
