@@ -500,6 +500,79 @@ def test_bounded_wait_reports_timeout_and_context_survives():
     plan.close()
 
 
+def test_batch_and_side_stream():
+    """B = 2 equals two B = 1 calls, and calls enqueued on a non-default stream give the same bits."""
+    cfg = CFG_MID128
+    plan = make_plan(cfg)
+    Q1, K1, V1 = tile_major_inputs(cfg, plan)
+    cfg2 = dict(cfg, seed=cfg["seed"] + 1)
+    Q2, K2, V2 = tile_major_inputs(cfg2, plan)
+    Q, K, V = (torch.cat([a, b], dim=0).contiguous() for a, b in ((Q1, Q2), (K1, K2), (V1, V2)))
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    _, _, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    plan.check_status()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    for b, (q, k, v) in enumerate(((Q1, K1, V1), (Q2, K2, V2))):
+        with torch.cuda.stream(side):
+            o, h, _ = plan.entropy_attn(q, k, v)
+            _, _, r = plan.budget_radius(h)
+            m, rp, ci, nz = plan.build_block_mask(r)
+            os_, _ = plan.sparse_attn(q, k, v, rp, ci)
+        side.synchronize()
+        assert torch.equal(o[0], O[b]) and torch.equal(h[0], H[b])
+        assert torch.equal(r[0], ridx[b]) and torch.equal(m[0], mask[b])
+        assert torch.equal(os_[0], Os[b])
+    plan.check_status()
+    plan.close()
+
+
+def test_largest_supported_sequence():
+    """NB = 2048 key blocks (262,144 tokens) is the largest sequence the attention calls take; one
+    more block is refused.  One head, sampled rows against the oracle."""
+    cfg = common.small_config(32, 64, 128, heads=1, head_dim=128, block=128, tile_h=8, tile_w=16, seed=91,
+                              s_lo=0.2, s_hi=5.0)
+    geo = common.oracle_geometry(cfg)
+    assert geo.NB == 2048
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    _, _, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    plan.check_status()
+    rng = np.random.default_rng(17)
+    rows = np.unique(np.concatenate([[0, geo.N - 1, geo.N // 2], rng.integers(0, geo.N, 9)])).astype(np.int32)
+    rows_t = torch.from_numpy(rows).long().to(DEV)
+    Qb, Kb, Vb = (workloads.bf16_bits(x[0, 0]) for x in (Q, K, V))
+    ref = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows)
+    common.assert_output(O[0, 0][rows_t], ref["O"], "dense at 262,144 tokens")
+    Hn = H[0, 0].cpu().numpy()
+    assert np.abs(Hn[rows] - ref["H_def"]).max() <= common.ENTROPY_ATOL
+    bud_ref, fragile = oracle.budget(Hn[None], geo.tau, geo.N)
+    ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)[0]
+    ridx_np = ridx[0, 0].cpu().numpy().view(np.uint16)
+    assert np.array_equal(ridx_np[~fragile[0]], ridx_ref[~fragile[0]]) and fragile.sum() <= 1
+    u_list = np.unique(rows // geo.block)
+    ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx_np, u_list=u_list)
+    assert np.array_equal(mask[0, 0].cpu().numpy()[u_list], ref_mask)
+    vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np, rows,
+                              ref_mask[np.searchsorted(u_list, rows // geo.block)], 0)
+    refs = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis)
+    common.assert_output(Os[0, 0][rows_t], refs["O"], "sparse at 262,144 tokens")
+    plan.close()
+    # one block more: the attention calls refuse, the integer stages still run
+    big = make_plan(cfg, n_text=1)
+    assert big.NB == 2049
+    z = torch.zeros(1, 1, big.N, 128, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(api().TraError) as e:
+        big.entropy_attn(z, z, z)
+    assert e.value.code == -2          # TRA_ERR_UNSUPPORTED
+    big.close()
+
+
 def test_attention_rejects_bad_arguments():
     a = api()
     plan = make_plan(CFG_TINY)
