@@ -158,15 +158,19 @@ int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* 
                          int64_t* nnz_out, int B, int heads, void* stream);
 
 /* Block-sparse attention (Eq. 16 as executed: Section 3.2, last paragraph, and "Limitations"):
- * softmax attention of each query over all valid keys of the retained key blocks of its block
- * row; retained blocks are evaluated in full, no token mask inside them.  A query whose block
- * row is empty gets O = 0.
+ * softmax attention of each query over the valid keys of the retained key blocks of its block row.
+ *   ridx == NULL: retained blocks are evaluated in full, no token mask inside them (what the
+ *                 paper's block-sparse execution does);
+ *   ridx != NULL: uint16 [B, heads, N] from tra_budget_radius; inside the retained blocks a video
+ *                 query additionally sees only the video keys inside its disk (the token mask of
+ *                 Eq. 15 on top of the block list); text keys and text queries are not masked.
+ * A query that is left with no visible key gets O = 0 and lse = -inf.
  *   row_ptr, col_idx: the CSR list written by tra_build_block_mask (reusable across calls:
- *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL, -inf for an empty
- *   row; formed from the bf16-rounded probabilities (absolute error up to about 4e-3). */
+ *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL; formed
+ *   from the bf16-rounded probabilities (absolute error up to about 4e-3). */
 int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
-                    const int32_t* row_ptr, const int32_t* col_idx, void* O, float* lse, int B,
-                    int heads, float sm_scale, void* stream);
+                    const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, void* O,
+                    float* lse, int B, int heads, float sm_scale, void* stream);
 
 #ifdef __cplusplus
 }

@@ -64,7 +64,7 @@ def _load():
     lib.tra_entropy_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
     lib.tra_budget_radius.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
     lib.tra_build_block_mask.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int64, vp, i32, i32, vp]
-    lib.tra_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
+    lib.tra_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
     return lib
 
 
@@ -251,8 +251,10 @@ class Plan:
                "tra_build_block_mask")
         return block_mask, row_ptr, col_idx, nnz
 
-    def sparse_attn(self, Q, K, V, row_ptr, col_idx, O=None, lse=None, want_lse=False, sm_scale=None):
-        """Block-sparse attention over the retained key blocks (tile-major inputs)."""
+    def sparse_attn(self, Q, K, V, row_ptr, col_idx, O=None, lse=None, want_lse=False, sm_scale=None,
+                    ridx=None):
+        """Block-sparse attention over the retained key blocks (tile-major inputs).  With ``ridx`` the
+        token mask of Eq. 15 is applied inside the retained blocks as well."""
         B, heads = self._bh(Q)
         if O is None:
             O = torch.empty_like(Q)
@@ -262,7 +264,8 @@ class Plan:
         bf = torch.bfloat16
         _check(_lib.tra_sparse_attn(self._h, _dev(Q, bf, "Q"), _dev(K, bf, "K"), _dev(V, bf, "V"),
                                     _dev(row_ptr, torch.int32, "row_ptr"),
-                                    _dev(col_idx, torch.int32, "col_idx"), _dev(O, bf, "O"),
+                                    _dev(col_idx, torch.int32, "col_idx"), _dev(ridx, torch.int16, "ridx"),
+                                    _dev(O, bf, "O"),
                                     _dev(lse, torch.float32, "lse"), B, heads, scale, _stream()),
                "tra_sparse_attn")
         return O, lse

@@ -290,14 +290,24 @@ struct SharedCtl {
 };
 static_assert(sizeof(SharedCtl) <= 2048, "control block");
 
+// Arguments of the optional token mask inside retained blocks (Eq. 15 applied on top of the block
+// list): packed coordinates of the video tokens (padded by one block), thresholds, candidate indices.
+struct TokenMaskArgs {
+  const uint32_t* coord_packed;
+  const int32_t* theta;
+  const uint16_t* ridx;
+  int n_video;
+  int T;
+};
+
 // ------------------------------------------------------------------------------------ kernel
-template <int D, int BN, bool kEntropy>
+template <int D, int BN, bool kEntropy, bool kTokenMask>
 __global__ void __launch_bounds__(kThreads, 1)
 tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ O,
                 float* __restrict__ entropy, float* __restrict__ lse,
                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, int N, int NB,
-                float scale_log2, int* __restrict__ status) {
+                float scale_log2, int* __restrict__ status, TokenMaskArgs tm) {
   using C = Cfg<D, BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -556,6 +566,18 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 
     float m = -INFINITY, l = 0.f, a = 0.f;
     float l_exact = 0.f;          // unrounded row sum (entropy kernels only)
+    // token mask: this query's coordinate and its row of the threshold table (video queries only)
+    bool tm_row = false;
+    int qx = 0, qy = 0, qt = 0;
+    const int32_t* th_row = nullptr;
+    if (kTokenMask && row < tm.n_video) {
+      const uint32_t c = tm.coord_packed[row];
+      qx = tra_coord_x(c);
+      qy = tra_coord_y(c);
+      qt = tra_coord_t(c);
+      th_row = tm.theta + (int)tm.ridx[(size_t)bh * N + row] * tm.T;
+      tm_row = true;
+    }
     uint32_t n = 0;               // key blocks this tile has processed
     uint32_t s_parity = 0;
     bool alive = true;
@@ -589,7 +611,30 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int j = 0; j < BN; ++j)
             if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
         }
+        if (kTokenMask && tm_row && active && v * BN < tm.n_video) {
+          // keys outside this query's disk at their frame distance do not exist for it (Eq. 15);
+          // text keys (index >= n_video) stay visible
+          const int k0 = v * BN;
+          const int kt0 = tra_coord_t(tm.coord_packed[k0]);
+          const int th0 = __ldg(th_row + abs(qt - kt0));
+          const int th1 = kt0 + 1 < tm.T ? __ldg(th_row + abs(qt - kt0 - 1)) : th0;
+          const uint4* kc4 = reinterpret_cast<const uint4*>(tm.coord_packed + k0);
+#pragma unroll
+          for (int j4 = 0; j4 < BN / 4; ++j4) {
+            const uint4 c4 = __ldg(kc4 + j4);
+            const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              const int j = j4 * 4 + q4;
+              const int dt = tra_coord_t(cs[q4]) - kt0;
+              const int th = dt == 0 ? th0 : (dt == 1 ? th1 : __ldg(th_row + abs(qt - kt0 - dt)));
+              const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
+              if (k0 + j < tm.n_video && dx * dx + dy * dy > th) sb[j] = __float_as_uint(-1e30f);
+            }
+          }
+        }
         float alpha = 1.f;
+        bool row_on = active;         // false also when the token mask leaves this row nothing here
         if (active) {
           float mx0 = __uint_as_float(sb[0]), mx1 = __uint_as_float(sb[1]);
 #pragma unroll
@@ -598,8 +643,10 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             mx1 = fmax3(mx1, __uint_as_float(sb[j + 2]), __uint_as_float(sb[j + 3]));
           }
           mx0 = fmax3(mx0, __uint_as_float(sb[BN - 2]), __uint_as_float(sb[BN - 1]));
-          const float m_blk = fmaxf(mx0, mx1) * scale_log2;
-          if (m_blk > m + kRescaleThreshold) {        // also the first block (m = -inf)
+          const float mx = fmaxf(mx0, mx1);
+          if (kTokenMask) row_on = mx > -1e29f;
+          const float m_blk = mx * scale_log2;
+          if (row_on && m_blk > m + kRescaleThreshold) {   // also the first block (m = -inf)
             alpha = ex2(m - m_blk);                   // 0 when m = -inf
             a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
             l *= alpha;
@@ -629,7 +676,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // probabilities (relative to m), row sum and entropy accumulator; P goes back to tensor
         // memory 32 keys at a time, and each 64-key half is announced to the MMA issuer on its own
         {
-          const float neg_m = active ? -m : 0.f;
+          const float neg_m = row_on ? -m : 0.f;
           const uint64_t scale2 = pack2(scale_log2, scale_log2), neg_m2 = pack2(neg_m, neg_m);
           uint64_t l2 = 0ull, a2 = 0ull, e2 = 0ull;      // pairs of partial sums
 #pragma unroll
@@ -770,30 +817,31 @@ int make_map(CUtensorMap* map, const void* base, int d, int N, long long BH, int
   return r == CUDA_SUCCESS ? TRA_OK : TRA_ERR_CUDA;
 }
 
-template <int D, int BN, bool kEntropy>
+template <int D, int BN, bool kEntropy, bool kTokenMask>
 int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O, float* entropy,
-           float* lse, const int32_t* row_ptr, const int32_t* col_idx, long long BH, float sm_scale,
-           cudaStream_t stream) {
+           float* lse, const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, long long BH,
+           float sm_scale, cudaStream_t stream) {
   using C = Cfg<D, BN>;
   CUtensorMap mq, mk, mv;
   int rc;
   if ((rc = make_map(&mq, Q, D, plan->S, BH, kTileM)) != TRA_OK) return rc;
   if ((rc = make_map(&mk, K, D, plan->S, BH, BN)) != TRA_OK) return rc;
   if ((rc = make_map(&mv, V, D, plan->S, BH, BN)) != TRA_OK) return rc;
-  auto kern = tra_attn_kernel<D, BN, kEntropy>;
+  auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask>;
+  TokenMaskArgs tm = {plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
   TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
   dim3 grid((unsigned)n_pairs, (unsigned)BH);
   kern<<<grid, kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, (__nv_bfloat16*)O, entropy, lse, row_ptr,
                                                   col_idx, plan->S, plan->NB, sm_scale * kLog2e,
-                                                  plan->d_status);
+                                                  plan->d_status, tm);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }
 
 int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O,
-                  float* entropy, float* lse, const int32_t* row_ptr, const int32_t* col_idx, int B,
-                  int heads, float sm_scale, void* stream_) {
+                  float* entropy, float* lse, const int32_t* row_ptr, const int32_t* col_idx,
+                  const uint16_t* ridx, int B, int heads, float sm_scale, void* stream_) {
   if (!plan || !Q || !K || !V || !O || B < 1 || heads < 1) return TRA_ERR_INVALID_ARG;
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O) & 127) return TRA_ERR_INVALID_ARG;
   if (!(sm_scale > 0.f)) return TRA_ERR_INVALID_ARG;
@@ -801,19 +849,23 @@ int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const vo
   if (BH > 65535 || plan->NB > 32 * kMaxBitmapWords) return TRA_ERR_UNSUPPORTED;
   cudaStream_t stream = (cudaStream_t)stream_;
   const int d = plan->cfg.head_dim, b = plan->cfg.block;
-  const bool ent = entropy != nullptr;
-  if (d == 128 && b == 128)
-    return ent ? launch<128, 128, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
-               : launch<128, 128, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
-  if (d == 64 && b == 64)
-    return ent ? launch<64, 64, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
-               : launch<64, 64, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
-  if (d == 64 && b == 128)
-    return ent ? launch<64, 128, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
-               : launch<64, 128, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
-  if (d == 128 && b == 64)
-    return ent ? launch<128, 64, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream)
-               : launch<128, 64, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, BH, sm_scale, stream);
+  const int variant = (entropy != nullptr ? 1 : 0) + (ridx != nullptr ? 2 : 0);   // never 3
+#define TRA_ATTN_CASE(DD, BB)                                                                          \
+  if (d == DD && b == BB) {                                                                            \
+    if (variant == 1)                                                                                  \
+      return launch<DD, BB, true, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, BH,   \
+                                         sm_scale, stream);                                            \
+    if (variant == 2)                                                                                  \
+      return launch<DD, BB, false, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, BH,   \
+                                         sm_scale, stream);                                            \
+    return launch<DD, BB, false, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, BH,    \
+                                        sm_scale, stream);                                             \
+  }
+  TRA_ATTN_CASE(128, 128)
+  TRA_ATTN_CASE(64, 64)
+  TRA_ATTN_CASE(64, 128)
+  TRA_ATTN_CASE(128, 64)
+#undef TRA_ATTN_CASE
   return TRA_ERR_UNSUPPORTED;
 }
 
@@ -843,12 +895,12 @@ extern "C" int tra_selftest_wait_timeout(tra_plan_t* plan, int limit_ms, void* s
 extern "C" int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
                                 void* O, float* entropy, float* lse, int B, int heads, float sm_scale,
                                 void* stream) {
-  return attn_dispatch(plan, Q, K, V, O, entropy, lse, nullptr, nullptr, B, heads, sm_scale, stream);
+  return attn_dispatch(plan, Q, K, V, O, entropy, lse, nullptr, nullptr, nullptr, B, heads, sm_scale, stream);
 }
 
 extern "C" int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
-                               const int32_t* row_ptr, const int32_t* col_idx, void* O, float* lse, int B,
-                               int heads, float sm_scale, void* stream) {
+                               const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, void* O,
+                               float* lse, int B, int heads, float sm_scale, void* stream) {
   if (!row_ptr || !col_idx) return TRA_ERR_INVALID_ARG;
-  return attn_dispatch(plan, Q, K, V, O, nullptr, lse, row_ptr, col_idx, B, heads, sm_scale, stream);
+  return attn_dispatch(plan, Q, K, V, O, nullptr, lse, row_ptr, col_idx, ridx, B, heads, sm_scale, stream);
 }

@@ -196,7 +196,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
     }
 
   // tile-major order and per-block boxes (Section 3.3)
-  std::vector<uint32_t> packed(p->N);
+  std::vector<uint32_t> packed(p->N + 128, 0u);   // padded by one block for vector loads past the end
   std::vector<int32_t> raster(p->N);
   std::vector<int32_t> tile_of_pos(p->N);
   {
@@ -244,7 +244,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
 
   // device tables
   const size_t count_elems = (size_t)p->N * nr;
-  bool ok = cudaMalloc(&p->d_coord_packed, sizeof(uint32_t) * p->N) == cudaSuccess &&
+  bool ok = cudaMalloc(&p->d_coord_packed, sizeof(uint32_t) * (p->N + 128)) == cudaSuccess &&
             cudaMalloc(&p->d_raster_of_pos, sizeof(int32_t) * p->N) == cudaSuccess &&
             cudaMalloc(&p->d_theta, sizeof(int32_t) * nr * T) == cudaSuccess &&
             cudaMalloc(&p->d_radii_f32, sizeof(float) * nr) == cudaSuccess &&
@@ -252,7 +252,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
             cudaMalloc(&p->d_boxes, sizeof(tra_block_boxes_t) * p->NB) == cudaSuccess &&
             cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess;
   ok = ok &&
-       cudaMemcpyAsync(p->d_coord_packed, packed.data(), sizeof(uint32_t) * p->N,
+       cudaMemcpyAsync(p->d_coord_packed, packed.data(), sizeof(uint32_t) * (p->N + 128),
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&
        cudaMemcpyAsync(p->d_raster_of_pos, raster.data(), sizeof(int32_t) * p->N,
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&

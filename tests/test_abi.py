@@ -38,4 +38,5 @@ def test_status_strings_and_null_arguments():
     assert lib.tra_plan_create(None, None, None) == -1
     assert lib.tra_plan_destroy(None) == -1
     assert lib.tra_budget_radius(None, None, None, None, None, 1, 1, None) == -1
+    assert lib.tra_sparse_attn(None, None, None, None, None, None, None, None, None, 1, 1, ctypes.c_float(1.0), None) == -1
     assert lib.tra_entropy_attn(None, None, None, None, None, None, None, 1, 1, ctypes.c_float(1.0), None) == -1

@@ -282,6 +282,47 @@ def test_sparse_attn_all_rows(cfg, kind):
     plan.close()
 
 
+@pytest.mark.parametrize("cfg,n_text", [(CFG_TINY, 0), (CFG_RAGGED64, 0), (CFG_RAGGED128, 0), (CFG_MID128, 0),
+                                        (CFG_RAGGED64, 50), (CFG_RAGGED128, 200)],
+                         ids=["tiny", "ragged64", "ragged128", "mid128", "ragged64+text", "ragged128+text"])
+@pytest.mark.parametrize("kind", ["entropy", "small", "uniform"])
+def test_sparse_attn_with_token_mask(cfg, n_text, kind):
+    """ridx passed to the sparse call: block list AND the token mask of Eq. 15 (oracle mode 1)."""
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg, n_text=n_text)
+    S, b = geo.N + n_text, geo.block
+    NB = (S + b - 1) // b
+    Qr, Kr, Vr = workloads.make_qkv(cfg, DEV)
+    if n_text:
+        Qr, Kr, Vr = workloads.append_text(Qr, Kr, Vr, cfg, n_text)
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    rv = random_ridx(geo, cfg["heads"], np.random.default_rng(31), kind)
+    ridx = np.full((cfg["heads"], S), geo.radii.size - 1, np.uint16)
+    ridx[:, : geo.N] = rv
+    ridx_t = torch.from_numpy(ridx.view(np.int16)).to(DEV)[None]
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx_t)
+    O, lse = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx_t, want_lse=True)
+    plan.check_status()
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(S)
+    n_empty = n_masked = 0
+    for h in range(cfg["heads"]):
+        ref_mask = oracle.block_vote(geo.coord, geo.T, b, geo.theta, ridx[h], u_list=np.arange(NB), n_text=n_text)
+        assert np.array_equal(mask[0, h].cpu().numpy(), ref_mask)
+        vis0 = oracle.visible_rows(geo.coord, geo.T, b, geo.theta, ridx[h], rows, ref_mask[rows // b], 0, n_text=n_text)
+        vis1 = oracle.visible_rows(geo.coord, geo.T, b, geo.theta, ridx[h], rows, ref_mask[rows // b], 1, n_text=n_text)
+        n_masked += int(vis0.sum() - vis1.sum())
+        ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis1)
+        common.assert_output(O[0, h], ref["O"], f"token-mask head {h}")
+        empty = ~vis1.astype(bool).any(axis=1)
+        n_empty += int(empty.sum())
+        assert np.all(O[0, h].float().cpu().numpy()[empty] == 0)
+        assert np.all(np.isneginf(lse[0, h].cpu().numpy()[empty]))
+    if kind == "uniform":
+        assert n_masked > 0                   # the token mask removed pairs the block list kept
+    plan.close()
+
+
 def test_sparse_attn_full_mask_equals_dense():
     # every block retained: the sparse call reproduces dense attention (full-support radius)
     cfg = CFG_RAGGED128
