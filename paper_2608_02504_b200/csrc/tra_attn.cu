@@ -619,17 +619,31 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const int th0 = __ldg(th_row + abs(qt - kt0));
           const int th1 = kt0 + 1 < tm.T ? __ldg(th_row + abs(qt - kt0 - 1)) : th0;
           const uint4* kc4 = reinterpret_cast<const uint4*>(tm.coord_packed + k0);
+          const bool one_frame = k0 + BN <= tm.n_video && tra_coord_t(tm.coord_packed[k0 + BN - 1]) == kt0;
+          if (one_frame) {              // the usual case: every key of the block in one frame
 #pragma unroll
-          for (int j4 = 0; j4 < BN / 4; ++j4) {
-            const uint4 c4 = __ldg(kc4 + j4);
-            const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
+            for (int j4 = 0; j4 < BN / 4; ++j4) {
+              const uint4 c4 = __ldg(kc4 + j4);
+              const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-              const int j = j4 * 4 + q4;
-              const int dt = tra_coord_t(cs[q4]) - kt0;
-              const int th = dt == 0 ? th0 : (dt == 1 ? th1 : __ldg(th_row + abs(qt - kt0 - dt)));
-              const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
-              if (k0 + j < tm.n_video && dx * dx + dy * dy > th) sb[j] = __float_as_uint(-1e30f);
+              for (int q4 = 0; q4 < 4; ++q4) {
+                const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
+                if (dx * dx + dy * dy > th0) sb[j4 * 4 + q4] = __float_as_uint(-1e30f);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j4 = 0; j4 < BN / 4; ++j4) {
+              const uint4 c4 = __ldg(kc4 + j4);
+              const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
+#pragma unroll
+              for (int q4 = 0; q4 < 4; ++q4) {
+                const int j = j4 * 4 + q4;
+                const int dt = tra_coord_t(cs[q4]) - kt0;
+                const int th = dt == 0 ? th0 : (dt == 1 ? th1 : __ldg(th_row + abs(qt - kt0 - dt)));
+                const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
+                if (k0 + j < tm.n_video && dx * dx + dy * dy > th) sb[j] = __float_as_uint(-1e30f);
+              }
             }
           }
         }
