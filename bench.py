@@ -44,9 +44,10 @@ METRIC = ("TRA hot-path effective TFLOP/s at 75.6K tokens (4*d*computed pairs / 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) per head of one sparse attention launch at the 75.6K-token shape, from
 # the ncu capture of a 4-head case summarised in profiles/attention_kernels_wan14b-720p_4heads.md
-# (234.4 MB + 59.3 MB for 4 heads); traffic grows in proportion to the head count.
-NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (234.363648e6 + 59.300864e6) / 4
-NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (233.931520e6 + 63.376128e6) / 4
+# (235.5 MB + 60.1 MB for 4 heads; 237.0 + 60.5 MB for the fused dense + entropy launch); traffic
+# grows in proportion to the head count.
+NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (235.540480e6 + 60.053248e6) / 4
+NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (236.979712e6 + 60.492544e6) / 4
 
 
 def load_peaks():
