@@ -78,6 +78,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait; false = gave up (abort flag raised by this or another thread).
 __device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                             int* status, unsigned long long limit_ns = kWaitLimitNs) {
+  // The global timer is slow to read, so it is consulted only after many failed polls (each
+  // try_wait already suspends the thread for a while): ordinary waits never touch it.
+#pragma unroll 1
+  for (uint32_t it = 0; it < 4096u; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = globaltimer_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -301,7 +306,8 @@ struct TokenMaskArgs {
 };
 
 // ------------------------------------------------------------------------------------ kernel
-template <int D, int BN, bool kEntropy, bool kTokenMask>
+// kDense: every query block attends to every key block (no block list; row_ptr is not read).
+template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense>
 __global__ void __launch_bounds__(kThreads, 1)
 tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ O,
@@ -331,8 +337,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
     for (int k = 0; k < 2; ++k) {
       mbar_init(smem_u32(&ctl->s_full[k]), 1);
-      mbar_init(smem_u32(&ctl->p_ready[k][0]), kTileM);
-      mbar_init(smem_u32(&ctl->p_ready[k][1]), kTileM);
+      mbar_init(smem_u32(&ctl->p_ready[k][0]), 4);     // one lane of each of the tile's four warps
+      mbar_init(smem_u32(&ctl->p_ready[k][1]), 4);
       mbar_init(smem_u32(&ctl->o_done[k]), 1);
     }
     mbar_init(smem_u32(&ctl->drain), 1);
@@ -348,16 +354,11 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   }
   for (int i = tid; i < 4 * kMaxBitmapWords; i += kThreads) (&ctl->bitmap[0][0])[i] = 0u;
   __syncthreads();
-  // key-block bitmaps of the query blocks this CTA holds
-  for (int g = 0; g < C::kBlocksPerCta; ++g) {
+  // key-block bitmaps of the query blocks this CTA holds (block-sparse launches only)
+  for (int g = 0; g < C::kBlocksPerCta && !kDense; ++g) {
     const int ub = pair * C::kBlocksPerCta + g;
     if (ub >= NB) continue;
-    if (row_ptr == nullptr) {
-      for (int w = tid; w < n_words; w += kThreads) {
-        int rem = NB - 32 * w;
-        ctl->bitmap[g][w] = rem >= 32 ? 0xffffffffu : ((1u << rem) - 1u);
-      }
-    } else {
+    {
       const long long r = (long long)bh * NB + ub;
       const int lo = row_ptr[r], hi = row_ptr[r + 1];
       for (int e = lo + tid; e < hi; e += kThreads) {
@@ -371,6 +372,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   tc_fence_after();
   const uint32_t tmem = ctl->tmem_base;
 
+  // dense launches: a tile takes part when its first query block exists
+  const bool tile1_on = pair * C::kBlocksPerCta + C::kGroups < NB;
+  const int n_outer = kDense ? 1 : n_words;   // dense launches walk 0 .. NB-1 in one inner loop
   // bitmap of a tile = union over its query blocks
   auto tile_word = [&](int k, int w) -> uint32_t {
     uint32_t x = ctl->bitmap[k * C::kGroups][w];
@@ -392,11 +396,17 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       int slot = 0;
       uint32_t phase = 0;
       bool alive = true;
-      for (int w = 0; w < n_words && alive; ++w) {
-        uint32_t bits = tile_word(0, w) | tile_word(1, w);
-        while (bits && alive) {
-          const int v = 32 * w + __ffs(bits) - 1;
-          bits &= bits - 1;
+      for (int w = 0; w < n_outer && alive; ++w) {
+        uint32_t bits = kDense ? 0u : (tile_word(0, w) | tile_word(1, w));
+        int v_dense = 0;
+        while ((kDense ? v_dense < NB : bits != 0u) && alive) {
+          int v;
+          if (kDense) {
+            v = v_dense++;
+          } else {
+            v = 32 * w + __ffs(bits) - 1;
+            bits &= bits - 1;
+          }
           for (int kv = 0; kv < 2; ++kv) {
             if (!mbar_wait(smem_u32(&ctl->kv_empty[slot]), phase ^ 1u, abort_flag, status)) {
               alive = false;
@@ -479,6 +489,13 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       int w = 0;
       uint32_t bits0 = 0, bits1 = 0;      // remaining bits of the current word, per tile
       auto next_entry = [&](bool& h0, bool& h1) -> bool {
+        if (kDense) {                       // w counts key blocks
+          if (w >= NB) return false;
+          ++w;
+          h0 = true;
+          h1 = tile1_on;
+          return true;
+        }
         while (true) {
           const uint32_t u = bits0 | bits1;
           if (u) {
@@ -582,14 +599,22 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     uint32_t s_parity = 0;
     bool alive = true;
 
-    for (int w = 0; w < n_words && alive; ++w) {
-      uint32_t bits = tile_word(k, w);
-      const uint32_t own_bits = ctl->bitmap[g_own][w];
-      while (bits) {
-        const uint32_t low = bits & (0u - bits);
-        bits &= ~low;
-        const int v = 32 * w + __ffs(low) - 1;
-        const bool active = (own_bits & low) != 0;
+    const int n_dense = (k == 0 || tile1_on) ? NB : 0;
+    for (int w = 0; w < n_outer && alive; ++w) {
+      uint32_t bits = kDense ? 0u : tile_word(k, w);
+      const uint32_t own_bits = kDense ? 0u : ctl->bitmap[g_own][w];
+      int v_dense = 0;
+      while (kDense ? v_dense < n_dense : bits != 0u) {
+        int v;
+        bool active = true;      // a tile that is one query block retains every block of its list
+        if (kDense) {
+          v = v_dense++;
+        } else {
+          const uint32_t low = bits & (0u - bits);
+          bits &= ~low;
+          v = 32 * w + __ffs(low) - 1;
+          if (C::kGroups > 1) active = (own_bits & low) != 0;
+        }
         const int col_limit = min(BN, N - v * BN);
 
         if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl->s_full[k]), s_parity, abort_flag, status))) {
@@ -724,7 +749,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             if (c & 1) {                      // a 64-key half of P is complete
               tmem_wait_st();
               tc_fence_before();
-              mbar_arrive(smem_u32(&ctl->p_ready[k][c >> 1]));
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&ctl->p_ready[k][c >> 1]));
             }
           }
           float lo, hi;
@@ -831,7 +857,7 @@ int make_map(CUtensorMap* map, const void* base, int d, int N, long long BH, int
   return r == CUDA_SUCCESS ? TRA_OK : TRA_ERR_CUDA;
 }
 
-template <int D, int BN, bool kEntropy, bool kTokenMask>
+template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense>
 int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O, float* entropy,
            float* lse, const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, long long BH,
            float sm_scale, cudaStream_t stream) {
@@ -841,7 +867,7 @@ int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, 
   if ((rc = make_map(&mq, Q, D, plan->S, BH, kTileM)) != TRA_OK) return rc;
   if ((rc = make_map(&mk, K, D, plan->S, BH, BN)) != TRA_OK) return rc;
   if ((rc = make_map(&mv, V, D, plan->S, BH, BN)) != TRA_OK) return rc;
-  auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask>;
+  auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense>;
   TokenMaskArgs tm = {plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
   TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
@@ -863,17 +889,22 @@ int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const vo
   if (BH > 65535 || plan->NB > 32 * kMaxBitmapWords) return TRA_ERR_UNSUPPORTED;
   cudaStream_t stream = (cudaStream_t)stream_;
   const int d = plan->cfg.head_dim, b = plan->cfg.block;
+  // entropy launches are dense, token-mask launches block-sparse; a plain launch may be either
   const int variant = (entropy != nullptr ? 1 : 0) + (ridx != nullptr ? 2 : 0);   // never 3
+  if ((variant == 1 && row_ptr != nullptr) || (variant == 2 && row_ptr == nullptr)) return TRA_ERR_INVALID_ARG;
 #define TRA_ATTN_CASE(DD, BB)                                                                          \
   if (d == DD && b == BB) {                                                                            \
     if (variant == 1)                                                                                  \
-      return launch<DD, BB, true, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, BH,   \
-                                         sm_scale, stream);                                            \
+      return launch<DD, BB, true, false, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, \
+                                               BH, sm_scale, stream);                                  \
     if (variant == 2)                                                                                  \
-      return launch<DD, BB, false, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, BH,   \
-                                         sm_scale, stream);                                            \
-    return launch<DD, BB, false, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, BH,    \
-                                        sm_scale, stream);                                             \
+      return launch<DD, BB, false, true, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx,      \
+                                                ridx, BH, sm_scale, stream);                           \
+    if (row_ptr == nullptr)                                                                            \
+      return launch<DD, BB, false, false, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx,      \
+                                                ridx, BH, sm_scale, stream);                           \
+    return launch<DD, BB, false, false, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, \
+                                               BH, sm_scale, stream);                                  \
   }
   TRA_ATTN_CASE(128, 128)
   TRA_ATTN_CASE(64, 64)
