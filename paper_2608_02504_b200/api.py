@@ -269,3 +269,99 @@ class Plan:
                                     _dev(lse, torch.float32, "lse"), B, heads, scale, _stream()),
                "tra_sparse_attn")
         return O, lse
+
+
+class HostPipeline:
+    """One pass of the hot path over tensors that live in pinned host memory.
+
+    The pass runs in groups of heads (heads are independent problems): while the kernels of group g
+    run, the inputs of group g + 1 travel to the device on a copy stream and the output of group
+    g - 1 travels back on another, so the PCIe time hides behind the kernels.  Every step of the
+    path (layout, dense attention + entropy, budget / radius, block vote, block-sparse attention,
+    layout back) is the library's kernels; this class only owns buffers, streams and events.
+
+    Inputs and outputs are bf16, raster token order, shape [1, heads, N, head_dim], pinned.
+    """
+
+    def __init__(self, plan: "Plan", heads: int, group: int = 8, device=None, sm_scale=None):
+        if heads < 1 or group < 1:
+            raise ValueError("heads and group must be positive")
+        self.plan, self.heads, self.group = plan, heads, min(group, heads)
+        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.dev = dev
+        g, N, d, NB = self.group, plan.N, plan.head_dim, plan.NB
+        bf = torch.bfloat16
+        self.scale = 1.0 / math.sqrt(d) if sm_scale is None else sm_scale
+        self.stage_in = [[torch.empty(1, g, N, d, dtype=bf, device=dev) for _ in range(3)] for _ in range(2)]
+        self.stage_out = [torch.empty(1, g, N, d, dtype=bf, device=dev) for _ in range(2)]
+        self.qkv = [torch.empty(1, g, N, d, dtype=bf, device=dev) for _ in range(3)]
+        self.o_dense = torch.empty(1, g, N, d, dtype=bf, device=dev)
+        self.o_sparse = torch.empty(1, g, N, d, dtype=bf, device=dev)
+        self.entropy = torch.empty(1, g, N, dtype=torch.float32, device=dev)
+        self.ridx = torch.empty(1, g, N, dtype=torch.int16, device=dev)
+        self.mask = torch.empty(1, g, NB, NB, dtype=torch.uint8, device=dev)
+        self.row_ptr = torch.empty(g * NB + 1, dtype=torch.int32, device=dev)
+        self.col_idx = torch.empty(g * NB * NB, dtype=torch.int32, device=dev)
+        self.nnz = torch.zeros(1, dtype=torch.int64, device=dev)
+        self.s_in, self.s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        self.launches_per_group = 10      # 3 gathers, dense, budget, vote + scan + fill, sparse, scatter
+
+    @staticmethod
+    def _check_host(t, shape, name):
+        if t.is_cuda or not t.is_pinned() or t.dtype != torch.bfloat16 or tuple(t.shape) != shape or \
+                not t.is_contiguous():
+            raise ValueError(f"{name}: expected a contiguous pinned bf16 host tensor of shape {shape}")
+
+    def run(self, Qh, Kh, Vh, Oh):
+        """Q, K, V (pinned host) -> O (pinned host).  Returns when every copy has been issued; the
+        caller synchronises (or records an event on the current stream, which waits for all of it)."""
+        plan, g = self.plan, self.group
+        shape = (1, self.heads, plan.N, plan.head_dim)
+        for t, name in ((Qh, "Q"), (Kh, "K"), (Vh, "V"), (Oh, "O")):
+            self._check_host(t, shape, name)
+        main = torch.cuda.current_stream(self.dev)
+        self.s_in.wait_stream(main)
+        self.s_out.wait_stream(main)
+        row_bytes = plan.head_dim * 2
+        groups = [(h0, min(g, self.heads - h0)) for h0 in range(0, self.heads, g)]
+        in_free = [None, None]            # events: the gathers that read staging buffer b are done
+        out_free = [None, None]           # events: the copy out of output buffer b is done
+        for i, (h0, n) in enumerate(groups):
+            b = i & 1
+            with torch.cuda.stream(self.s_in):
+                if in_free[b] is not None:
+                    self.s_in.wait_event(in_free[b])
+                for dst, src in zip(self.stage_in[b], (Qh, Kh, Vh)):
+                    dst[:, :n].copy_(src[:, h0:h0 + n], non_blocking=True)
+                ready = torch.cuda.Event()
+                ready.record(self.s_in)
+            main.wait_event(ready)
+            vp = ctypes.c_void_p
+            for src, dst in zip(self.stage_in[b], self.qkv):
+                _check(_lib.tra_tile_major_gather(plan._h, vp(src.data_ptr()), vp(dst.data_ptr()), n, row_bytes,
+                                                  _stream(main)), "tra_tile_major_gather")
+            in_free[b] = torch.cuda.Event()
+            in_free[b].record(main)
+            Q, K, V = (t[:, :n] for t in self.qkv)
+            plan.entropy_attn(Q, K, V, O=self.o_dense[:, :n], entropy=self.entropy[:, :n])
+            plan.budget_radius(self.entropy[:, :n], ridx=self.ridx[:, :n], want_budget=False, want_radius=False)
+            plan.build_block_mask(self.ridx[:, :n], block_mask=self.mask[:, :n],
+                                  row_ptr=self.row_ptr[: n * plan.NB + 1],
+                                  col_idx=self.col_idx[: n * plan.NB * plan.NB], nnz=self.nnz)
+            plan.sparse_attn(Q, K, V, self.row_ptr[: n * plan.NB + 1], self.col_idx[: n * plan.NB * plan.NB],
+                             O=self.o_sparse[:, :n])
+            if out_free[b] is not None:
+                main.wait_event(out_free[b])
+            _check(_lib.tra_tile_major_scatter(plan._h, vp(self.o_sparse.data_ptr()),
+                                               vp(self.stage_out[b].data_ptr()), n, row_bytes, _stream(main)),
+                   "tra_tile_major_scatter")
+            done = torch.cuda.Event()
+            done.record(main)
+            with torch.cuda.stream(self.s_out):
+                self.s_out.wait_event(done)
+                Oh[:, h0:h0 + n].copy_(self.stage_out[b][:, :n], non_blocking=True)
+                out_free[b] = torch.cuda.Event()
+                out_free[b].record(self.s_out)
+        main.wait_stream(self.s_out)
+        main.wait_stream(self.s_in)
+        return len(groups) * self.launches_per_group

@@ -570,6 +570,33 @@ def test_batch_and_side_stream():
     plan.close()
 
 
+def test_host_pipeline_matches_device_path():
+    """The head-group pipeline over pinned host tensors (copies overlapped with kernels) returns the
+    bits of the one-shot device path, with a ragged last group and with one group."""
+    cfg = dict(CFG_MID128, heads=5)
+    plan = make_plan(cfg)
+    Qr, Kr, Vr = workloads.make_qkv(cfg, "cuda")
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    _, H, _ = plan.entropy_attn(Q, K, V)
+    _, _, ridx = plan.budget_radius(H)
+    _, row_ptr, col_idx, _ = plan.build_block_mask(ridx)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    expect = plan.tile_major_scatter(Os).cpu()
+    host = [t.cpu().pin_memory() for t in (Qr, Kr, Vr)]
+    for group in (2, 8):
+        pipe = api().HostPipeline(plan, cfg["heads"], group=group)
+        out = torch.zeros(expect.shape, dtype=torch.bfloat16).pin_memory()
+        for _ in range(2):                      # the second run reuses every buffer
+            launches = pipe.run(host[0], host[1], host[2], out)
+            torch.cuda.synchronize()
+            assert torch.equal(out, expect)
+        assert launches == 10 * -(-cfg["heads"] // min(group, cfg["heads"]))
+    with pytest.raises(ValueError):
+        pipe.run(Qr, host[1], host[2], out)     # a device tensor where a pinned host tensor belongs
+    plan.check_status()
+    plan.close()
+
+
 def test_largest_supported_sequence():
     """NB = 2048 key blocks (262,144 tokens) is the largest sequence the attention calls take; one
     more block is refused.  One head, sampled rows against the oracle."""
