@@ -44,10 +44,10 @@ METRIC = ("TRA hot-path effective TFLOP/s at 75.6K tokens (4*d*computed pairs / 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) per head of one sparse attention launch at the 75.6K-token shape, from
 # the ncu capture of a 4-head case summarised in profiles/attention_kernels_wan14b-720p_4heads.md
-# (235.5 MB + 60.1 MB for 4 heads; 237.0 + 60.5 MB for the fused dense + entropy launch); traffic
+# (234.2 MB + 58.7 MB for 4 heads; 237.0 + 62.1 MB for the fused dense + entropy launch); traffic
 # grows in proportion to the head count.
-NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (235.540480e6 + 60.053248e6) / 4
-NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (236.979712e6 + 60.492544e6) / 4
+NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (234.245888e6 + 58.742272e6) / 4
+NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (236.973056e6 + 62.136832e6) / 4
 
 
 def load_peaks():
@@ -320,10 +320,10 @@ def run_ours(args):
                 "peak_source": peak_note, "flops_per_launch": flops, "launch_ms": round(seconds * 1e3, 4)}
 
     full_shape = args.config == "wan14b-720p"
-    roofline = attn_roofline("tra_attn_kernel<128,128,true> (dense attention + entropy)", tf_dense,
+    roofline = attn_roofline("tra_attn_kernel<128,128,entropy,-,dense> (dense attention + entropy)", tf_dense,
                              4.0 * d * pairs_dense, t_dense,
                              NCU_DENSE_TRAFFIC_BYTES_PER_HEAD * heads if full_shape else None)
-    roofline_sparse = attn_roofline("tra_attn_kernel<128,128,false> (block-sparse attention)", tf_sparse,
+    roofline_sparse = attn_roofline("tra_attn_kernel<128,128,-,-,block list> (block-sparse attention)", tf_sparse,
                                     4.0 * d * pairs_sparse, t_sparse,
                                     NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD * heads if full_shape else None)
 
