@@ -373,6 +373,11 @@ def run_ours(args):
         K.copy_(k_keep)
         del q_keep, k_keep
 
+    # ---- the other shapes the paper measures on (same pass, stage times only) ------------------
+    other = None
+    if args.other_workloads and rank == 0 and args.config == "wan14b-720p" and args.heads is None:
+        other = [run_other_workload(api, name, dev, peak_tf) for name in ("wan1.3b-480p", "hunyuan-720p")]
+
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region --------
     e2e = None
     if rank == 0 or world > 1:
@@ -396,7 +401,7 @@ def run_ours(args):
                        "l2": "inputs larger than L2 (Q/K/V/O are 774 MB each)"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "roofline_sparse": roofline_sparse, "stages": stages,
-            "tau_sweep": tau_sweep, "schedule": schedule, "cpu_baseline": cpu_baseline,
+            "tau_sweep": tau_sweep, "other_workloads": other, "schedule": schedule, "cpu_baseline": cpu_baseline,
             "paper_context": "paper: 1.56-2.05x end-to-end speedup at 9-19% retained interactions on one H200",
             "wall_s_timed_region": round(wall_s, 3),
         }
@@ -452,6 +457,61 @@ def run_schedule(cfg, plan, api, dev, bufs, n_steps, n_warm, refresh_every=0):
             "sparse_step_ms": round(float(np.mean(per_step[n_warm:])), 3),
             "retained_block_density": round(computed_pairs(mask, N, block) / (heads * float(N) * N), 4),
             "drift": "Q and K: x_t = x_{t-1} + 0.05 N(0,1) on the fp32 state; V fixed"}
+
+
+def run_other_workload(api, name, dev, peak_tf, reps=2):
+    """One of the other shapes the paper measures on (stage times of the same pass, 1 warm-up +
+    `reps` timed passes): ms per layer, TFLOP/s on computed pairs, retained density, speedup."""
+    cfg = dict(workloads.CONFIGS[name])
+    N, d, heads, block = workloads.num_tokens(cfg), cfg["head_dim"], cfg["heads"], cfg["block"]
+    plan = api.Plan.from_config(cfg)
+    Qr, Kr, Vr = workloads.make_qkv(cfg, dev)
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    del Qr, Kr, Vr
+    O = torch.empty_like(Q)
+    H = torch.empty(1, heads, N, dtype=torch.float32, device=dev)
+    ridx = torch.empty(1, heads, N, dtype=torch.int16, device=dev)
+    bufs = None
+    names = ("dense_entropy", "budget_radius", "block_mask", "sparse", "dense_plain")
+    ms = {k: [] for k in names}
+    for it in range(1 + reps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(6)]
+        ev[0].record()
+        plan.entropy_attn(Q, K, V, O=O, entropy=H)
+        ev[1].record()
+        plan.budget_radius(H, ridx=ridx, want_budget=False, want_radius=False)
+        ev[2].record()
+        if bufs is None:
+            bufs = plan.build_block_mask(ridx)
+        else:
+            plan.build_block_mask(ridx, *bufs)
+        ev[3].record()
+        plan.sparse_attn(Q, K, V, bufs[1], bufs[2], O=O)
+        ev[4].record()
+        plan.entropy_attn(Q, K, V, O=O, want_entropy=False)
+        ev[5].record()
+        torch.cuda.synchronize()
+        if it == 0:
+            plan.check_status()
+            continue
+        for i, k in enumerate(names):
+            ms[k].append(ev[i].elapsed_time(ev[i + 1]))
+    plan.check_status()
+    t = {k: float(np.mean(v)) for k, v in ms.items()}
+    pairs_sparse = computed_pairs(bufs[0], N, block)
+    pairs_dense = float(heads) * N * N
+    tf = lambda pairs, msec: 4.0 * d * pairs / (msec * 1e-3) / 1e12
+    out = {"workload": name, "tokens": N, "heads": heads, "gamma": cfg["gamma"], "tau": cfg["tau"],
+           "ms": {k: round(v, 4) for k, v in t.items()},
+           "dense_entropy_tflops": round(tf(pairs_dense, t["dense_entropy"]), 1),
+           "sparse_tflops": round(tf(pairs_sparse, t["sparse"]), 1),
+           "sparse_frac_of_peak": round(tf(pairs_sparse, t["sparse"]) / peak_tf, 4),
+           "block_density": round(pairs_sparse / pairs_dense, 4),
+           "speedup_sparse_vs_dense_plain": round(t["dense_plain"] / t["sparse"], 3),
+           "mask_radius_overhead_frac_of_sparse_layer": round(
+               (t["budget_radius"] + t["block_mask"]) / (t["sparse"] + t["budget_radius"] + t["block_mask"]), 4)}
+    plan.close()
+    return out
 
 
 def run_e2e(args, api, plan, src_dev, O_raster, flops_step, world, dev, group=8):
@@ -576,6 +636,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-schedule", dest="schedule", action="store_false")
     ap.add_argument("--no-tau-sweep", dest="tau_sweep", action="store_false")
+    ap.add_argument("--no-other-workloads", dest="other_workloads", action="store_false",
+                    help="skip the Wan2.1-1.3B and HunyuanVideo shapes reported next to the main workload")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
