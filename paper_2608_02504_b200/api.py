@@ -283,10 +283,13 @@ class HostPipeline:
     Inputs and outputs are bf16, raster token order, shape [1, heads, N, head_dim], pinned.
     """
 
-    def __init__(self, plan: "Plan", heads: int, group: int = 8, device=None, sm_scale=None):
-        if heads < 1 or group < 1:
-            raise ValueError("heads and group must be positive")
+    def __init__(self, plan: "Plan", heads: int, group: int = 8, device=None, sm_scale=None, first_group=None):
+        """``first_group`` (default ``group``): heads in the first group; a small first group lets the
+        kernels start while most of the input is still on its way."""
+        if heads < 1 or group < 1 or (first_group is not None and first_group < 1):
+            raise ValueError("heads, group and first_group must be positive")
         self.plan, self.heads, self.group = plan, heads, min(group, heads)
+        self.first_group = self.group if first_group is None else min(first_group, self.group)
         dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
         self.dev = dev
         g, N, d, NB = self.group, plan.N, plan.head_dim, plan.NB
@@ -323,7 +326,11 @@ class HostPipeline:
         self.s_in.wait_stream(main)
         self.s_out.wait_stream(main)
         row_bytes = plan.head_dim * 2
-        groups = [(h0, min(g, self.heads - h0)) for h0 in range(0, self.heads, g)]
+        groups, h0 = [], 0
+        while h0 < self.heads:
+            n = min(self.first_group if h0 == 0 else g, self.heads - h0)
+            groups.append((h0, n))
+            h0 += n
         in_free = [None, None]            # events: the gathers that read staging buffer b are done
         out_free = [None, None]           # events: the copy out of output buffer b is done
         for i, (h0, n) in enumerate(groups):

@@ -583,14 +583,15 @@ def test_host_pipeline_matches_device_path():
     Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
     expect = plan.tile_major_scatter(Os).cpu()
     host = [t.cpu().pin_memory() for t in (Qr, Kr, Vr)]
-    for group in (2, 8):
-        pipe = api().HostPipeline(plan, cfg["heads"], group=group)
+    for group, first in ((2, None), (8, None), (3, 1)):
+        pipe = api().HostPipeline(plan, cfg["heads"], group=group, first_group=first)
         out = torch.zeros(expect.shape, dtype=torch.bfloat16).pin_memory()
         for _ in range(2):                      # the second run reuses every buffer
             launches = pipe.run(host[0], host[1], host[2], out)
             torch.cuda.synchronize()
             assert torch.equal(out, expect)
-        assert launches == 10 * -(-cfg["heads"] // min(group, cfg["heads"]))
+        n_groups = -(-cfg["heads"] // min(group, cfg["heads"])) if first is None else 1 + -(-(cfg["heads"] - first) // group)
+        assert launches == 10 * n_groups
     with pytest.raises(ValueError):
         pipe.run(Qr, host[1], host[2], out)     # a device tensor where a pinned host tensor belongs
     plan.check_status()
