@@ -242,6 +242,16 @@ __device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+// floor(sqrt(n)) for 0 <= n < 2^22 with no conversion instruction (conversions share the
+// special-function unit with ex2): n + 0.5 is formed from the 2^23 bit pattern, sqrt.approx of it
+// stays at least 0.25 / sqrt(n) away from every integer, and adding 2^23 - 0.5 rounds it down into
+// the low mantissa bits.
+__device__ __forceinline__ int tra_isqrt_small_nocvt(int n) {
+  const float f = __uint_as_float(0x4B000000u | (uint32_t)n) - 8388607.5f;      // n + 0.5, exact
+  float r;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(f));
+  return (int)(__float_as_uint(r + 8388607.5f) & 0x7FFFFFu);
+}
 // bf16x2 with `lo` in the low half
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   uint32_t d;
@@ -298,6 +308,7 @@ static_assert(sizeof(SharedCtl) <= 2048, "control block");
 // Arguments of the optional token mask inside retained blocks (Eq. 15 applied on top of the block
 // list): packed coordinates of the video tokens (padded by one block), thresholds, candidate indices.
 struct TokenMaskArgs {
+  const uint32_t* slice;          // one word per 16 positions (plan table): run of one frame row or 0
   const uint32_t* coord_packed;
   const int32_t* theta;
   const uint16_t* ridx;
@@ -645,7 +656,37 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const int th1 = kt0 + 1 < tm.T ? __ldg(th_row + abs(qt - kt0 - 1)) : th0;
           const uint4* kc4 = reinterpret_cast<const uint4*>(tm.coord_packed + k0);
           const bool one_frame = k0 + BN <= tm.n_video && tra_coord_t(tm.coord_packed[k0 + BN - 1]) == kt0;
-          if (one_frame) {              // the usual case: every key of the block in one frame
+          // 16-key slices of the block; the usual case: each is 16 consecutive x of one frame row
+          uint32_t sl[BN / 16];
+#pragma unroll
+          for (int q = 0; q < BN / 64; ++q) {
+            const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(tm.slice + (k0 >> 4)) + q);
+            sl[4 * q] = w4.x;
+            sl[4 * q + 1] = w4.y;
+            sl[4 * q + 2] = w4.z;
+            sl[4 * q + 3] = w4.w;
+          }
+          uint32_t all_runs = sl[0];
+#pragma unroll
+          for (int q = 1; q < BN / 16; ++q) all_runs &= sl[q];
+          if (all_runs & (1u << 30)) {
+            // A key (x0 + j, ys) is inside the disk iff |x0 + j - qx| <= w with
+            // w = floor(sqrt(theta - (ys - qy)^2)): one square root per slice, then an unsigned
+            // range test per key:  0 <= j + (x0 - qx + w) <= 2 w.
+#pragma unroll
+            for (int q = 0; q < BN / 16; ++q) {
+              const int ts = (int)((sl[q] >> 20) & 1023u), dts = ts - kt0;
+              const int th = dts == 0 ? th0 : (dts == 1 ? th1 : __ldg(th_row + abs(qt - ts)));
+              const int dy = tra_coord_y(sl[q]) - qy;
+              const int rem = th - dy * dy;
+              const int w = tra_isqrt_small_nocvt(max(rem, 0));
+              const uint32_t base = rem < 0 ? 0x40000000u : (uint32_t)(w + tra_coord_x(sl[q]) - qx);
+              const uint32_t span = (uint32_t)(2 * w);
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (base + (uint32_t)j > span) sb[q * 16 + j] = __float_as_uint(-1e30f);
+            }
+          } else if (one_frame) {       // every key of the block in one frame, some slice not a row run
 #pragma unroll
             for (int j4 = 0; j4 < BN / 4; ++j4) {
               const uint4 c4 = __ldg(kc4 + j4);
@@ -868,7 +909,7 @@ int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, 
   if ((rc = make_map(&mk, K, D, plan->S, BH, BN)) != TRA_OK) return rc;
   if ((rc = make_map(&mv, V, D, plan->S, BH, BN)) != TRA_OK) return rc;
   auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense>;
-  TokenMaskArgs tm = {plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
+  TokenMaskArgs tm = {plan->d_slice, plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
   TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
   dim3 grid((unsigned)n_pairs, (unsigned)BH);

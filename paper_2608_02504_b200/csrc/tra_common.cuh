@@ -34,6 +34,9 @@ struct tra_plan {
   int32_t* h_coord;   // [N][3]
   // device tables
   uint32_t* d_coord_packed;       // [N]  x | y << 10 | t << 20   per tile-major position
+  uint32_t* d_slice;              // [NB * block / 16, padded to 8]  one word per 16 consecutive positions:
+                                  // x0 | y << 10 | t << 20 | 1 << 30 when they are 16 video tokens of
+                                  // one frame and one row with x = x0 .. x0 + 15, else 0
   int32_t* d_raster_of_pos;       // [N]
   int32_t* d_theta;               // [n_radii][T]
   float* d_radii_f32;             // [n_radii]

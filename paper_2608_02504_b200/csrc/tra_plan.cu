@@ -96,6 +96,7 @@ static void tra_plan_free(tra_plan* p) {
   free(p->h_theta);
   free(p->h_coord);
   cudaFree(p->d_coord_packed);
+  cudaFree(p->d_slice);
   cudaFree(p->d_raster_of_pos);
   cudaFree(p->d_theta);
   cudaFree(p->d_radii_f32);
@@ -242,9 +243,25 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
     boxes[u] = bb;
   }
 
+  // 16-position slices that are a run of one frame row (the token mask inside blocks tests such a
+  // slice as an x-interval)
+  const size_t n_slice = (((size_t)p->NB * cfg->block / 16) + 7) & ~(size_t)7;
+  std::vector<uint32_t> slices(n_slice, 0u);
+  for (size_t si = 0; si < n_slice; ++si) {
+    const long long p0 = (long long)si * 16;
+    if (p0 + 15 >= p->N) continue;
+    const int t = p->h_coord[3 * p0], y = p->h_coord[3 * p0 + 1], x = p->h_coord[3 * p0 + 2];
+    bool run = true;
+    for (int j = 1; j < 16 && run; ++j)
+      run = p->h_coord[3 * (p0 + j)] == t && p->h_coord[3 * (p0 + j) + 1] == y &&
+            p->h_coord[3 * (p0 + j) + 2] == x + j;
+    if (run) slices[si] = tra_pack_coord(t, y, x) | (1u << 30);
+  }
+
   // device tables
   const size_t count_elems = (size_t)p->N * nr;
   bool ok = cudaMalloc(&p->d_coord_packed, sizeof(uint32_t) * (p->N + 128)) == cudaSuccess &&
+            cudaMalloc(&p->d_slice, sizeof(uint32_t) * n_slice) == cudaSuccess &&
             cudaMalloc(&p->d_raster_of_pos, sizeof(int32_t) * p->N) == cudaSuccess &&
             cudaMalloc(&p->d_theta, sizeof(int32_t) * nr * T) == cudaSuccess &&
             cudaMalloc(&p->d_radii_f32, sizeof(float) * nr) == cudaSuccess &&
@@ -254,6 +271,8 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   ok = ok &&
        cudaMemcpyAsync(p->d_coord_packed, packed.data(), sizeof(uint32_t) * (p->N + 128),
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+       cudaMemcpyAsync(p->d_slice, slices.data(), sizeof(uint32_t) * n_slice, cudaMemcpyHostToDevice,
+                       stream) == cudaSuccess &&
        cudaMemcpyAsync(p->d_raster_of_pos, raster.data(), sizeof(int32_t) * p->N,
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&
        cudaMemcpyAsync(p->d_theta, p->h_theta, sizeof(int32_t) * nr * T, cudaMemcpyHostToDevice,

@@ -389,7 +389,7 @@ def sampled_rows(geo, rng, n_random):
 def test_full_size_sampled_rows(name, heads_checked, n_random):
     """At the BASELINE shapes, all heads resident, in the launch configuration the benchmark times:
     sampled (head, row) pairs of dense attention + entropy, the integer stages of their block
-    rows, and sparse attention.  Rows cover the first / last blocks and the ragged tail."""
+    rows, sparse attention, and sparse attention with the token mask inside the blocks.  Rows cover the first / last blocks and the ragged tail."""
     cfg = workloads.CONFIGS[name]
     geo = common.oracle_geometry(cfg)
     plan = make_plan(cfg)
@@ -398,6 +398,7 @@ def test_full_size_sampled_rows(name, heads_checked, n_random):
     budget, radius, ridx = plan.budget_radius(H)
     mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
     Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    Ot, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx)      # token mask inside the blocks
     plan.check_status()
     rng = np.random.default_rng(15)
     for h in heads_checked:
@@ -424,6 +425,10 @@ def test_full_size_sampled_rows(name, heads_checked, n_random):
         vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np, rows, block_rows, 0)
         refs = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis)
         common.assert_output(Os[0, h][rows_t], refs["O"], f"sparse {name} h{h}")
+        vis1 = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np, rows, block_rows, 1)
+        assert vis1.sum() < vis.sum()
+        reft = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis1)
+        common.assert_output(Ot[0, h][rows_t], reft["O"], f"token mask {name} h{h}")
     # CSR of every head is the ascending list of the mask the same call wrote
     m = mask[0].reshape(-1, geo.NB).bool()
     counts = m.sum(dim=1)
