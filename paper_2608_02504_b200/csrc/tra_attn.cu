@@ -15,7 +15,9 @@
 // tile overwrites the first half of its S columns and feeds the PV MMA straight from tensor memory.
 // The two tiles alternate on the tensor pipe (PV_k(e) then S_k(e+1)) while the other tile's
 // softmax runs.  The key-block list of the CTA is the union of the lists of the query blocks it
-// holds; a tile skips the MMAs of a key block none of its query blocks retains.
+// holds; a tile skips the MMAs of a key block none of its query blocks retains.  Dense launches
+// (kDense) have no list and count key blocks instead.  With kTokenMask the softmax threads also
+// remove, inside every retained block, the keys outside their query's disk (Eq. 15).
 //
 // Online softmax state per row, in the base-2 domain (t = s * sm_scale * log2 e):
 //   m  running reference maximum (raised only when the new maximum exceeds it by more than 8,
