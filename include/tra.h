@@ -172,6 +172,31 @@ int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const 
                     const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, void* O,
                     float* lse, int B, int heads, float sm_scale, void* stream);
 
+/* ---- the whole pass over HOST tensors (the paper has no counterpart: plumbing around the calls
+ * above for callers whose Q, K, V and O live in host memory) ----------------------------- */
+
+/* One pass of the hot path — tile-major layout, dense attention + entropy, budget / radius, block
+ * mask, block-sparse attention (retained blocks in full), layout back — over
+ *   Q_host, K_host, V_host : HOST pointers, bf16 [heads, S, head_dim], RASTER token order (read),
+ *   O_host                 : HOST pointer, same shape and order (written): the block-sparse output.
+ * Heads are independent problems, so the pass runs in groups of `group` heads (the first group
+ * holds `first_group` <= group heads, so that the kernels start early); the host-to-device copy of
+ * the next group and the device-to-host copy of the previous one run on two copy streams owned by
+ * the plan while the kernels of the current group run on `stream`.  Pinned (page-locked) host
+ * memory is needed for the copies to overlap; pageable memory works but serialises.
+ *   workspace : DEVICE memory, 256-byte aligned, at least tra_hot_path_host_workspace_bytes(plan,
+ *               group) bytes; owned by the caller, free to reuse once `stream` has passed the call.
+ * The call allocates no device memory (it creates the plan's two copy streams on its first use and
+ * short-lived events).  It returns after enqueueing; `stream` completes after the last copy in
+ * either direction, so synchronising `stream` (or an event recorded on it) makes O_host valid.
+ * Calls that share a plan or a workspace must be ordered on `stream`.
+ * Errors: TRA_ERR_INVALID_ARG (NULL / misaligned pointer, non-positive count or scale),
+ * TRA_ERR_CAPACITY (workspace too small), TRA_ERR_CUDA; kernel-side errors as for the four calls. */
+size_t tra_hot_path_host_workspace_bytes(const tra_plan_t* plan, int group);
+int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const void* K_host, const void* V_host,
+                      void* O_host, void* workspace, size_t workspace_bytes, int heads, int group,
+                      int first_group, float sm_scale, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -27,6 +27,7 @@ EXPORTS = [
     "tra_plan_num_radii", "tra_plan_tables", "tra_plan_count_table", "tra_plan_status",
     "tra_status_string", "tra_selftest_wait_timeout", "tra_tile_major_gather", "tra_tile_major_scatter",
     "tra_entropy_attn", "tra_budget_radius", "tra_build_block_mask", "tra_sparse_attn",
+    "tra_hot_path_host_workspace_bytes", "tra_hot_path_host",
 ]
 
 
@@ -58,6 +59,9 @@ def _load():
     lib.tra_plan_status.argtypes = [vp, vp]
     lib.tra_status_string.argtypes = [i32]
     lib.tra_selftest_wait_timeout.argtypes = [vp, i32, vp]
+    lib.tra_hot_path_host_workspace_bytes.argtypes = [vp, i32]
+    lib.tra_hot_path_host_workspace_bytes.restype = ctypes.c_size_t
+    lib.tra_hot_path_host.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_size_t, i32, i32, i32, f32, vp]
     lib.tra_status_string.restype = ctypes.c_char_p
     lib.tra_tile_major_gather.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.tra_tile_major_scatter.argtypes = [vp, vp, vp, i32, i32, vp]
@@ -272,13 +276,12 @@ class Plan:
 
 
 class HostPipeline:
-    """One pass of the hot path over tensors that live in pinned host memory.
+    """One pass of the hot path over tensors that live in pinned host memory (``tra_hot_path_host``).
 
-    The pass runs in groups of heads (heads are independent problems): while the kernels of group g
-    run, the inputs of group g + 1 travel to the device on a copy stream and the output of group
-    g - 1 travels back on another, so the PCIe time hides behind the kernels.  Every step of the
-    path (layout, dense attention + entropy, budget / radius, block vote, block-sparse attention,
-    layout back) is the library's kernels; this class only owns buffers, streams and events.
+    The library runs the pass in groups of heads (heads are independent problems): while the kernels
+    of group g run, the inputs of group g + 1 travel to the device on a copy stream and the output of
+    group g - 1 travels back on another, so the PCIe time hides behind the kernels.  This class only
+    owns the device workspace the call needs.
 
     Inputs and outputs are bf16, raster token order, shape [1, heads, N, head_dim], pinned.
     """
@@ -290,24 +293,13 @@ class HostPipeline:
             raise ValueError("heads, group and first_group must be positive")
         self.plan, self.heads, self.group = plan, heads, min(group, heads)
         self.first_group = self.group if first_group is None else min(first_group, self.group)
-        dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
-        self.dev = dev
-        g, N, d, NB = self.group, plan.N, plan.head_dim, plan.NB
-        bf = torch.bfloat16
-        self.scale = 1.0 / math.sqrt(d) if sm_scale is None else sm_scale
-        self.stage_in = [[torch.empty(1, g, N, d, dtype=bf, device=dev) for _ in range(3)] for _ in range(2)]
-        self.stage_out = [torch.empty(1, g, N, d, dtype=bf, device=dev) for _ in range(2)]
-        self.qkv = [torch.empty(1, g, N, d, dtype=bf, device=dev) for _ in range(3)]
-        self.o_dense = torch.empty(1, g, N, d, dtype=bf, device=dev)
-        self.o_sparse = torch.empty(1, g, N, d, dtype=bf, device=dev)
-        self.entropy = torch.empty(1, g, N, dtype=torch.float32, device=dev)
-        self.ridx = torch.empty(1, g, N, dtype=torch.int16, device=dev)
-        self.mask = torch.empty(1, g, NB, NB, dtype=torch.uint8, device=dev)
-        self.row_ptr = torch.empty(g * NB + 1, dtype=torch.int32, device=dev)
-        self.col_idx = torch.empty(g * NB * NB, dtype=torch.int32, device=dev)
-        self.nnz = torch.zeros(1, dtype=torch.int64, device=dev)
-        self.s_in, self.s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        self.dev = torch.device("cuda", torch.cuda.current_device()) if device is None else torch.device(device)
+        self.scale = 1.0 / math.sqrt(plan.head_dim) if sm_scale is None else sm_scale
+        self.workspace_bytes = int(_lib.tra_hot_path_host_workspace_bytes(plan._h, self.group))
+        self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.dev)
+        self._ws_ptr = (self.workspace.data_ptr() + 255) & ~255
         self.launches_per_group = 10      # 3 gathers, dense, budget, vote + scan + fill, sparse, scatter
+        self.n_groups = 1 + -(-(heads - self.first_group) // self.group)
 
     @staticmethod
     def _check_host(t, shape, name):
@@ -316,59 +308,14 @@ class HostPipeline:
             raise ValueError(f"{name}: expected a contiguous pinned bf16 host tensor of shape {shape}")
 
     def run(self, Qh, Kh, Vh, Oh):
-        """Q, K, V (pinned host) -> O (pinned host).  Returns when every copy has been issued; the
-        caller synchronises (or records an event on the current stream, which waits for all of it)."""
-        plan, g = self.plan, self.group
-        shape = (1, self.heads, plan.N, plan.head_dim)
+        """Q, K, V (pinned host) -> O (pinned host).  Returns the number of kernels launched once every
+        copy and kernel has been enqueued; synchronise the current stream before reading ``Oh``."""
+        shape = (1, self.heads, self.plan.N, self.plan.head_dim)
         for t, name in ((Qh, "Q"), (Kh, "K"), (Vh, "V"), (Oh, "O")):
             self._check_host(t, shape, name)
-        main = torch.cuda.current_stream(self.dev)
-        self.s_in.wait_stream(main)
-        self.s_out.wait_stream(main)
-        row_bytes = plan.head_dim * 2
-        groups, h0 = [], 0
-        while h0 < self.heads:
-            n = min(self.first_group if h0 == 0 else g, self.heads - h0)
-            groups.append((h0, n))
-            h0 += n
-        in_free = [None, None]            # events: the gathers that read staging buffer b are done
-        out_free = [None, None]           # events: the copy out of output buffer b is done
-        for i, (h0, n) in enumerate(groups):
-            b = i & 1
-            with torch.cuda.stream(self.s_in):
-                if in_free[b] is not None:
-                    self.s_in.wait_event(in_free[b])
-                for dst, src in zip(self.stage_in[b], (Qh, Kh, Vh)):
-                    dst[:, :n].copy_(src[:, h0:h0 + n], non_blocking=True)
-                ready = torch.cuda.Event()
-                ready.record(self.s_in)
-            main.wait_event(ready)
-            vp = ctypes.c_void_p
-            for src, dst in zip(self.stage_in[b], self.qkv):
-                _check(_lib.tra_tile_major_gather(plan._h, vp(src.data_ptr()), vp(dst.data_ptr()), n, row_bytes,
-                                                  _stream(main)), "tra_tile_major_gather")
-            in_free[b] = torch.cuda.Event()
-            in_free[b].record(main)
-            Q, K, V = (t[:, :n] for t in self.qkv)
-            plan.entropy_attn(Q, K, V, O=self.o_dense[:, :n], entropy=self.entropy[:, :n])
-            plan.budget_radius(self.entropy[:, :n], ridx=self.ridx[:, :n], want_budget=False, want_radius=False)
-            plan.build_block_mask(self.ridx[:, :n], block_mask=self.mask[:, :n],
-                                  row_ptr=self.row_ptr[: n * plan.NB + 1],
-                                  col_idx=self.col_idx[: n * plan.NB * plan.NB], nnz=self.nnz)
-            plan.sparse_attn(Q, K, V, self.row_ptr[: n * plan.NB + 1], self.col_idx[: n * plan.NB * plan.NB],
-                             O=self.o_sparse[:, :n])
-            if out_free[b] is not None:
-                main.wait_event(out_free[b])
-            _check(_lib.tra_tile_major_scatter(plan._h, vp(self.o_sparse.data_ptr()),
-                                               vp(self.stage_out[b].data_ptr()), n, row_bytes, _stream(main)),
-                   "tra_tile_major_scatter")
-            done = torch.cuda.Event()
-            done.record(main)
-            with torch.cuda.stream(self.s_out):
-                self.s_out.wait_event(done)
-                Oh[:, h0:h0 + n].copy_(self.stage_out[b][:, :n], non_blocking=True)
-                out_free[b] = torch.cuda.Event()
-                out_free[b].record(self.s_out)
-        main.wait_stream(self.s_out)
-        main.wait_stream(self.s_in)
-        return len(groups) * self.launches_per_group
+        vp = ctypes.c_void_p
+        _check(_lib.tra_hot_path_host(self.plan._h, vp(Qh.data_ptr()), vp(Kh.data_ptr()), vp(Vh.data_ptr()),
+                                      vp(Oh.data_ptr()), vp(self._ws_ptr), self.workspace_bytes, self.heads,
+                                      self.group, self.first_group, self.scale,
+                                      _stream(torch.cuda.current_stream(self.dev))), "tra_hot_path_host")
+        return self.n_groups * self.launches_per_group

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtra_b200.so")
-SOURCES = ["tra_plan.cu", "tra_radius.cu", "tra_mask.cu", "tra_attn.cu"]
+SOURCES = ["tra_plan.cu", "tra_radius.cu", "tra_mask.cu", "tra_attn.cu", "tra_host.cu"]
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

@@ -508,21 +508,22 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           h0 = true;
           h1 = tile1_on;
           return true;
-        }
-        while (true) {
-          const uint32_t u = bits0 | bits1;
-          if (u) {
-            const uint32_t low = u & (0u - u);
-            h0 = (bits0 & low) != 0;
-            h1 = (bits1 & low) != 0;
-            bits0 &= ~low;
-            bits1 &= ~low;
-            return true;
+        } else {
+          while (true) {
+            const uint32_t u = bits0 | bits1;
+            if (u) {
+              const uint32_t low = u & (0u - u);
+              h0 = (bits0 & low) != 0;
+              h1 = (bits1 & low) != 0;
+              bits0 &= ~low;
+              bits1 &= ~low;
+              return true;
+            }
+            if (w >= n_words) return false;
+            bits0 = tile_word(0, w);
+            bits1 = tile_word(1, w);
+            ++w;
           }
-          if (w >= n_words) return false;
-          bits0 = tile_word(0, w);
-          bits1 = tile_word(1, w);
-          ++w;
         }
       };
 

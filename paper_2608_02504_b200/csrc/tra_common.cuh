@@ -43,6 +43,8 @@ struct tra_plan {
   uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)
   tra_block_boxes_t* d_boxes;     // [NB]
   int* d_status;                  // device status word
+  // copy streams of tra_hot_path_host, created on its first call with this plan
+  cudaStream_t copy_in, copy_out;
 };
 
 __host__ __device__ inline uint32_t tra_pack_coord(int t, int y, int x) {

@@ -103,6 +103,8 @@ static void tra_plan_free(tra_plan* p) {
   cudaFree(p->d_counts);
   cudaFree(p->d_boxes);
   cudaFree(p->d_status);
+  if (p->copy_in) cudaStreamDestroy(p->copy_in);
+  if (p->copy_out) cudaStreamDestroy(p->copy_out);
   delete p;
 }
 

@@ -599,6 +599,16 @@ def test_host_pipeline_matches_device_path():
         assert launches == 10 * n_groups
     with pytest.raises(ValueError):
         pipe.run(Qr, host[1], host[2], out)     # a device tensor where a pinned host tensor belongs
+    # the C entry point refuses a workspace that is too small or misaligned, before any work
+    import ctypes
+    lib, vp = api()._lib, ctypes.c_void_p
+    args = [vp(t.data_ptr()) for t in host] + [vp(out.data_ptr())]
+    need = pipe.workspace_bytes
+    assert lib.tra_hot_path_host(plan._h, *args, vp(pipe._ws_ptr), need - 1, cfg["heads"], pipe.group, 1, 1.0,
+                                 None) == -3
+    assert lib.tra_hot_path_host(plan._h, *args, vp(pipe._ws_ptr + 16), need, cfg["heads"], pipe.group, 1, 1.0,
+                                 None) == -1
+    assert lib.tra_hot_path_host(plan._h, *args, vp(pipe._ws_ptr), need, 0, pipe.group, 1, 1.0, None) == -1
     plan.check_status()
     plan.close()
 
