@@ -165,6 +165,63 @@ def test_block_mask_bit_exact(cfg, kind):
         plan.close()
 
 
+def _random_geometries(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        block = int(rng.choice([64, 128]))
+        th, tw = int(rng.choice([1, 2, 4, 8, 16])), int(rng.choice([4, 8, 16, 32]))
+        out.append(common.small_config(int(rng.integers(1, 7)), int(rng.integers(3, 34)), int(rng.integers(3, 50)),
+                                       heads=2, head_dim=64, block=block, tile_h=th, tile_w=tw,
+                                       gamma=float(rng.choice([0.0, 0.0513, 0.6, 0.95, 2.0])),
+                                       tau=float(rng.choice([0.3, 0.5, 0.9, 1.0])), seed=200 + i))
+    return out
+
+
+@pytest.mark.parametrize("cfg", _random_geometries(10, 5), ids=lambda c: f"{c['T']}x{c['H']}x{c['W']}-b{c['block']}-"
+                                                                         f"t{c['tile_h']}x{c['tile_w']}")
+def test_random_geometries_integer_stages_and_token_mask(cfg):
+    """Seeded random grids, tile shapes, decay rates and target masses: plan tables, budget, radius,
+    block mask and active-block list bit for bit; sparse attention with the token mask against the
+    oracle (its slices are row runs for some of these tile shapes and per-key tests for others)."""
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    radii, theta, coord = plan.tables()
+    assert np.array_equal(radii, geo.radii) and np.array_equal(theta, geo.theta) and np.array_equal(coord, geo.coord)
+    assert np.array_equal(plan.count_table(), geo.counts)
+    rng = np.random.default_rng(cfg["seed"])
+    heads = cfg["heads"]
+    H = rng.uniform(0.0, math.log(max(geo.N, 2)), (1, heads, geo.N)).astype(np.float32)
+    bud_ref, fragile = oracle.budget(H[0], geo.tau, geo.N)
+    ridx_ref = oracle.select_radius(bud_ref, geo.coord, geo.H, geo.W, geo.counts)
+    budget, radius, ridx = plan.budget_radius(torch.from_numpy(H).to(DEV))
+    ok = ~fragile
+    assert fragile.sum() <= 2
+    assert np.array_equal(budget.cpu().numpy()[0][ok], bud_ref[ok])
+    assert np.array_equal(ridx.cpu().numpy().view(np.uint16)[0][ok], ridx_ref[ok])
+    # masks and lists from the oracle's candidate indices
+    ridx_t = torch.from_numpy(ridx_ref.astype(np.uint16).view(np.int16)).to(DEV)[None]
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx_t)
+    plan.check_status()
+    ref = np.stack([oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx_ref[h]) for h in range(heads)])
+    assert np.array_equal(mask.cpu().numpy()[0], ref)
+    rp, ci = oracle.csr_from_block_mask(ref)
+    assert int(nnz.item()) == rp[-1]
+    assert np.array_equal(row_ptr.cpu().numpy().astype(np.int64), rp)
+    assert np.array_equal(col_idx.cpu().numpy()[: rp[-1]], ci)
+    # token mask inside the retained blocks
+    Q, K, V = tile_major_inputs(cfg, plan)
+    O, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx_t)
+    plan.check_status()
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(geo.N)
+    for h in range(heads):
+        vis1 = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_ref[h], rows, ref[h][rows // geo.block], 1)
+        r = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis1)
+        common.assert_output(O[0, h], r["O"], f"token-mask head {h}")
+    plan.close()
+
+
 def test_block_mask_capacity_error_is_reported():
     cfg = CFG_TINY
     geo = common.oracle_geometry(cfg)
