@@ -28,7 +28,8 @@
 //    memory; a prefix sum along each row turns it into the counts (a disk that covers the whole
 //    frame is only counted once, a disk that covers a whole row skips the square root).  Every undecided key block
 //    then reads the counts of its own keys in that frame (c_j by definition) and accumulates
-//    its numbers of reached and of high columns.
+//    its numbers of reached and of high columns.  When the query block lies in one frame t0 the
+//    frames t0 - k and t0 + k see the same thresholds, so one field serves both.
 // The outcome equals the unpruned vote bit for bit.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ int tra_isqrt_small(int n) {
@@ -151,13 +152,13 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   __syncthreads();
 
   // ---- 2. count field of every frame that holds an undecided key block ---------------------
-  for (int f = 0; f < T; ++f) {
-    if (!s_frame_needed[f]) continue;                   // uniform across the CTA
+  // builds the field for the frame distance dist(thread) -> |f - t_i| of every query
+  auto build_field = [&](auto dist_of_query) {
     for (int i = tid; i < H * Wp; i += TRA_MASK_THREADS) s_diff[i] = 0;
     if (tid == 0) s_whole = 0;
     __syncthreads();
     if (tid < nq) {
-      const int th = __ldg(theta + qr * T + abs(qt - f));
+      const int th = __ldg(theta + qr * T + dist_of_query());
       const int far_x = max(qx, W - 1 - qx), far_y = max(qy, H - 1 - qy);
       if (th >= far_x * far_x + far_y * far_y) {
         atomicAdd(&s_whole, 1);                       // the disk covers the whole frame
@@ -196,7 +197,9 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       }
     }
     __syncthreads();
-    // undecided key blocks with tokens in this frame: one warp per block
+  };
+  // undecided key blocks with tokens in frame f read the field: one warp per block
+  auto count_frame = [&](int f) {
     const int whole = s_whole;                         // queries whose disk covers every key of the frame
     const int p_begin = f * HW, p_end = min(N, (f + 1) * HW);
     const int v_first = p_begin / b, v_last = (p_end - 1) / b;     // video blocks only: p_end <= N
@@ -219,7 +222,31 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
         s_hi[v] = (uint16_t)(s_hi[v] + hi);
       }
     }
-    __syncthreads();
+  };
+  // A query block that lies in one frame t0 sees frames t0 - k and t0 + k at the same distance:
+  // their fields are the same, so one field serves both.
+  bool one_frame = s_ubox.n_box > 0;
+  for (int iu = 0; iu < s_ubox.n_box; ++iu)
+    one_frame = one_frame && s_ubox.box[iu].t0 == s_ubox.box[0].t0 && s_ubox.box[iu].t1 == s_ubox.box[0].t0;
+  if (one_frame) {
+    const int t0 = s_ubox.box[0].t0;
+    for (int k = 0; k < T; ++k) {
+      const int fa = t0 - k, fb = t0 + k;
+      const bool need_a = fa >= 0 && s_frame_needed[fa];
+      const bool need_b = k > 0 && fb < T && s_frame_needed[fb];
+      if (!need_a && !need_b) continue;                 // uniform across the CTA
+      build_field([&]() { return k; });
+      if (need_a) count_frame(fa);
+      if (need_b) count_frame(fb);
+      __syncthreads();
+    }
+  } else {
+    for (int f = 0; f < T; ++f) {
+      if (!s_frame_needed[f]) continue;                 // uniform across the CTA
+      build_field([&]() { return abs(qt - f); });
+      count_frame(f);
+      __syncthreads();
+    }
   }
 
   // ---- 3. votes of the undecided key blocks -------------------------------------------------
