@@ -296,10 +296,9 @@ struct Cfg {
 struct SharedCtl {
   uint64_t q_full;
   uint64_t kv_full[6];
-  uint64_t kv_empty[6];
+  uint64_t kv_release[4];   // ring slots are handed back in release events (see the MMA warp)
   uint64_t s_full[2];
   uint64_t p_ready[2][2];   // [tile][64-key half of the block]
-  uint64_t o_done[2];
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
@@ -346,13 +345,12 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     mbar_init(smem_u32(&ctl->q_full), 1);
     for (int i = 0; i < C::kSlots; ++i) {
       mbar_init(smem_u32(&ctl->kv_full[i]), 1);
-      mbar_init(smem_u32(&ctl->kv_empty[i]), 1);
     }
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&ctl->kv_release[i]), 1);
     for (int k = 0; k < 2; ++k) {
       mbar_init(smem_u32(&ctl->s_full[k]), 1);
       mbar_init(smem_u32(&ctl->p_ready[k][0]), 4);     // one lane of each of the tile's four warps
       mbar_init(smem_u32(&ctl->p_ready[k][1]), 4);
-      mbar_init(smem_u32(&ctl->o_done[k]), 1);
     }
     mbar_init(smem_u32(&ctl->drain), 1);
     ctl->abort_flag = 0;
@@ -407,8 +405,12 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tma_load_3d(smem_u32(sQ + k * C::kQTileBytes + a * C::kQAtomBytes), &map_q, qbar, a * 64,
                       q_base + k * kTileM, bh);
       int slot = 0;
-      uint32_t phase = 0;
       bool alive = true;
+      // Loads go K0, V0, K1, V1, ... into consecutive slots.  The MMA warp hands slots back in
+      // release events: event 0 frees K0, event e + 1 frees V_e and K_(e+1) with one commit, so load
+      // j is freed by event (j + 1) / 2.  Event r arrives on kv_release[r % 4] as its (r / 4)-th
+      // completion; the producer has always passed event r before event r + 4 can be committed.
+      int n_load = 0;
       for (int w = 0; w < n_outer && alive; ++w) {
         uint32_t bits = kDense ? 0u : (tile_word(0, w) | tile_word(1, w));
         int v_dense = 0;
@@ -421,20 +423,21 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             bits &= bits - 1;
           }
           for (int kv = 0; kv < 2; ++kv) {
-            if (!mbar_wait(smem_u32(&ctl->kv_empty[slot]), phase ^ 1u, abort_flag, status)) {
-              alive = false;
-              break;
+            if (n_load >= C::kSlots) {          // the slot's previous load must have been released
+              const int r = (n_load - C::kSlots + 1) >> 1;
+              if (!mbar_wait(smem_u32(&ctl->kv_release[r & 3]), (uint32_t)(r >> 2) & 1u, abort_flag, status)) {
+                alive = false;
+                break;
+              }
             }
+            ++n_load;
             const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
             mbar_expect_tx(fbar, C::kSlotBytes);
             const CUtensorMap* map = kv == 0 ? &map_k : &map_v;
             for (int a = 0; a < C::kAtoms; ++a)
               tma_load_3d(smem_u32(sKV + slot * C::kSlotBytes + a * C::kKVAtomBytes), map, fbar, a * 64,
                           v * BN, bh);
-            if (++slot == C::kSlots) {
-              slot = 0;
-              phase ^= 1u;
-            }
+            if (++slot == C::kSlots) slot = 0;
           }
         }
       }
@@ -458,7 +461,6 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);
       const uint32_t v_lo0 = desc_lo(smem_u32(sKV), C::kKVAtomBytes);
       const uint32_t s_full_bar[2] = {smem_u32(&ctl->s_full[0]), smem_u32(&ctl->s_full[1])};
-      const uint32_t o_done_bar[2] = {smem_u32(&ctl->o_done[0]), smem_u32(&ctl->o_done[1])};
 
       auto issue_s = [&](int k, int kslot) {
         const uint32_t qa = q_lo[k];
@@ -487,7 +489,6 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           for (int kk = half * 4; kk < half * 4 + 4; ++kk)
             tc_mma_ts(d, pa + kk * 8, va + kk * (2048 >> 4), kHi, kIdescPV, (n_pv[k] > 0 || kk > 0) ? 1u : 0u);
         }
-        tc_commit(o_done_bar[k]);
         ++n_pv[k];
         return true;
       };
@@ -536,10 +537,11 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tc_fence_after();
           for (int k = 0; k < 2; ++k)
             if (h[k]) issue_s(k, slot);
-          tc_commit(smem_u32(&ctl->kv_empty[slot]));
+          tc_commit(smem_u32(&ctl->kv_release[0]));        // release event 0: K0
           advance();
         }
       }
+      uint32_t n_release = 1;
       while (have && alive) {
         const int vslot = slot;
         const uint32_t vphase = phase;
@@ -569,11 +571,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
         }
         if (!alive) break;
-        tc_commit(smem_u32(&ctl->kv_empty[vslot]));
-        if (have_next) {
-          tc_commit(smem_u32(&ctl->kv_empty[kslot]));
-          advance();
-        }
+        tc_commit(smem_u32(&ctl->kv_release[n_release & 3u]));   // V of this entry and K of the next
+        ++n_release;
+        if (have_next) advance();
         have = have_next;
         h[0] = hn[0];
         h[1] = hn[1];
@@ -740,12 +740,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         // rescale the O accumulator when some row of this warp raised its reference maximum
         const bool warp_rescale = __any_sync(0xffffffffu, alpha != 1.f) && n > 0;
         if (warp_rescale) {
-          if (!__all_sync(0xffffffffu,
-                          mbar_wait(smem_u32(&ctl->o_done[k]), (n - 1u) & 1u, abort_flag, status))) {
-            alive = false;
-            break;
-          }
-          tc_fence_after();
+          // PV(n-1) of this tile has retired: the S the thread just read was issued behind it on
+          // the same in-order pipe, and the commit that announced S covers every earlier MMA
 #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t o[32];
@@ -813,9 +809,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     }
 
     // ---- epilogue: O = o / l, entropy, lse ------------------------------------------------
+    // the MMA warp commits `drain` behind its last MMA: every PV of both tiles has retired then
     if (alive && n > 0)
-      alive = __all_sync(0xffffffffu,
-                         mbar_wait(smem_u32(&ctl->o_done[k]), (n - 1u) & 1u, abort_flag, status));
+      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl->drain), 0u, abort_flag, status));
     if (alive) {
       tc_fence_after();
       const float inv_l = l > 0.f ? 1.f / l : 0.f;
