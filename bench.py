@@ -44,10 +44,10 @@ METRIC = ("TRA hot-path effective TFLOP/s at 75.6K tokens (4*d*computed pairs / 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # DRAM bytes (read + write) per head of one sparse attention launch at the 75.6K-token shape, from
 # the ncu capture of a 4-head case summarised in profiles/attention_kernels_wan14b-720p_4heads.md
-# (234.2 MB + 58.7 MB for 4 heads; 237.0 + 62.1 MB for the fused dense + entropy launch); traffic
+# (234.4 MB + 61.1 MB for 4 heads; 237.1 + 62.2 MB for the fused dense + entropy launch); traffic
 # grows in proportion to the head count.
-NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (234.245888e6 + 58.742272e6) / 4
-NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (236.973056e6 + 62.136832e6) / 4
+NCU_SPARSE_TRAFFIC_BYTES_PER_HEAD = (234.363136e6 + 61.101568e6) / 4
+NCU_DENSE_TRAFFIC_BYTES_PER_HEAD = (237.128448e6 + 62.174464e6) / 4
 
 
 def load_peaks():
