@@ -247,7 +247,7 @@ def run_ours(args):
     stage_ms = {}
     for i, name in enumerate(stage_names):
         vals = [ev[k][i].elapsed_time(ev[k][i + 1]) for k in range(args.steps)]
-        stage_ms[name] = {"mean": float(np.mean(vals)), "min": float(np.min(vals))}
+        stage_ms[name] = {"mean": float(np.mean(vals)), "min": float(np.min(vals)), "median": float(np.median(vals))}
 
     pairs_sparse = computed_pairs(mask, N, block)
     pairs_dense = float(heads) * N * N
@@ -293,6 +293,7 @@ def run_ours(args):
     stages = {
         "ms": {k: round(v["mean"], 4) for k, v in stage_ms.items()},
         "ms_min": {k: round(v["min"], 4) for k, v in stage_ms.items()},
+        "ms_median": {k: round(v["median"], 4) for k, v in stage_ms.items()},
         "dense_plain_ms": round(t_plain * 1e3, 4),
         "dense_plain_tflops": round(4.0 * d * pairs_dense / t_plain / 1e12, 2),
         "dense_entropy_tflops": round(tf_dense, 2),
