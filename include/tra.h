@@ -164,6 +164,10 @@ int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* 
  *   ridx != NULL: uint16 [B, heads, N] from tra_budget_radius; inside the retained blocks a video
  *                 query additionally sees only the video keys inside its disk (the token mask of
  *                 Eq. 15 on top of the block list); text keys and text queries are not masked.
+ *   row_ptr == NULL and col_idx == NULL (only with ridx != NULL): Eq. 16 itself, no block list — a
+ *                 video query sees exactly the video keys inside its disk, text keys and text
+ *                 queries are not masked.  The kernel finds the key blocks a query block can reach
+ *                 from the plan's block boxes; no [heads, NB, NB] mask is needed.
  * A query that is left with no visible key gets O = 0 and lse = -inf.
  *   row_ptr, col_idx: the CSR list written by tra_build_block_mask (reusable across calls:
  *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL; formed

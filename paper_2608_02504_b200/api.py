@@ -258,7 +258,8 @@ class Plan:
     def sparse_attn(self, Q, K, V, row_ptr, col_idx, O=None, lse=None, want_lse=False, sm_scale=None,
                     ridx=None):
         """Block-sparse attention over the retained key blocks (tile-major inputs).  With ``ridx`` the
-        token mask of Eq. 15 is applied inside the retained blocks as well."""
+        token mask of Eq. 15 is applied inside the retained blocks as well; with ``ridx`` and
+        ``row_ptr = col_idx = None`` the call evaluates Eq. 16 itself (token mask alone, no block list)."""
         B, heads = self._bh(Q)
         if O is None:
             O = torch.empty_like(Q)

@@ -302,6 +302,7 @@ struct SharedCtl {
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
+  int rmax[4];              // largest candidate index among the video queries of each query block
   uint32_t bitmap[4][kMaxBitmapWords];
 };
 static_assert(sizeof(SharedCtl) <= 2048, "control block");
@@ -309,6 +310,7 @@ static_assert(sizeof(SharedCtl) <= 2048, "control block");
 // Arguments of the optional token mask inside retained blocks (Eq. 15 applied on top of the block
 // list): packed coordinates of the video tokens (padded by one block), thresholds, candidate indices.
 struct TokenMaskArgs {
+  const tra_block_boxes_t* boxes; // per-block boxes (plan table), for launches without a block list
   const uint32_t* slice;          // one word per 16 positions (plan table): run of one frame row or 0
   const uint32_t* coord_packed;
   const int32_t* theta;
@@ -364,9 +366,43 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   for (int i = tid; i < 4 * kMaxBitmapWords; i += kThreads) (&ctl->bitmap[0][0])[i] = 0u;
+  if (tid < 4) ctl->rmax[tid] = -1;
   __syncthreads();
+  // Token-mask launch without a block list (Eq. 16 itself): the key blocks a query block can reach
+  // at all, from the block boxes and the largest candidate index among its queries — a superset
+  // of the blocks that hold a visible key; the token mask inside the kernel does the rest.
+  const bool geometric_list = kTokenMask && row_ptr == nullptr;
+  if (geometric_list) {
+    for (int i = tid; i < 2 * kTileM; i += kThreads) {
+      const int row = q_base + i;
+      if (row < tm.n_video) atomicMax(&ctl->rmax[i / BN], (int)tm.ridx[(size_t)bh * N + row]);
+    }
+    __syncthreads();
+    for (int g = 0; g < C::kBlocksPerCta; ++g) {
+      const int ub = pair * C::kBlocksPerCta + g;
+      if (ub >= NB) continue;
+      const bool q_text = (ub + 1) * BN > tm.n_video;        // holds a text query: sees every key
+      const int rmax = ctl->rmax[g];
+      const tra_block_boxes_t ubx = tm.boxes[ub];
+      for (int v = tid; v < NB; v += kThreads) {
+        bool on = q_text || (v + 1) * BN > tm.n_video;         // text keys are always visible
+        if (!on && rmax >= 0) {
+          const tra_block_boxes_t vb = tm.boxes[v];
+          for (int iu = 0; iu < ubx.n_box && !on; ++iu)
+            for (int iv = 0; iv < vb.n_box && !on; ++iv) {
+              const tra_box_t a = ubx.box[iu], c = vb.box[iv];
+              const int dt_min = max(0, max(a.t0 - c.t1, c.t0 - a.t1));
+              const int gy = max(0, max(a.y0 - c.y1, c.y0 - a.y1));
+              const int gx = max(0, max(a.x0 - c.x1, c.x0 - a.x1));
+              on = tm.theta[rmax * tm.T + dt_min] >= gy * gy + gx * gx;
+            }
+        }
+        if (on) atomicOr(&ctl->bitmap[g][v >> 5], 1u << (v & 31));
+      }
+    }
+  }
   // key-block bitmaps of the query blocks this CTA holds (block-sparse launches only)
-  for (int g = 0; g < C::kBlocksPerCta && !kDense; ++g) {
+  for (int g = 0; g < C::kBlocksPerCta && !kDense && !geometric_list; ++g) {
     const int ub = pair * C::kBlocksPerCta + g;
     if (ub >= NB) continue;
     {
@@ -908,7 +944,7 @@ int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, 
   if ((rc = make_map(&mk, K, D, plan->S, BH, BN)) != TRA_OK) return rc;
   if ((rc = make_map(&mv, V, D, plan->S, BH, BN)) != TRA_OK) return rc;
   auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense>;
-  TokenMaskArgs tm = {plan->d_slice, plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
+  TokenMaskArgs tm = {plan->d_boxes, plan->d_slice, plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
   TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
   const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
   dim3 grid((unsigned)n_pairs, (unsigned)BH);
@@ -931,7 +967,7 @@ int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const vo
   const int d = plan->cfg.head_dim, b = plan->cfg.block;
   // entropy launches are dense, token-mask launches block-sparse; a plain launch may be either
   const int variant = (entropy != nullptr ? 1 : 0) + (ridx != nullptr ? 2 : 0);   // never 3
-  if ((variant == 1 && row_ptr != nullptr) || (variant == 2 && row_ptr == nullptr)) return TRA_ERR_INVALID_ARG;
+  if (variant == 1 && row_ptr != nullptr) return TRA_ERR_INVALID_ARG;
 #define TRA_ATTN_CASE(DD, BB)                                                                          \
   if (d == DD && b == BB) {                                                                            \
     if (variant == 1)                                                                                  \
@@ -986,6 +1022,7 @@ extern "C" int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const voi
 extern "C" int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
                                const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, void* O,
                                float* lse, int B, int heads, float sm_scale, void* stream) {
-  if (!row_ptr || !col_idx) return TRA_ERR_INVALID_ARG;
+  // a block list, or (with ridx) none at all: Eq. 16 itself
+  if ((row_ptr == nullptr) != (col_idx == nullptr) || (!row_ptr && !ridx)) return TRA_ERR_INVALID_ARG;
   return attn_dispatch(plan, Q, K, V, O, nullptr, lse, row_ptr, col_idx, ridx, B, heads, sm_scale, stream);
 }

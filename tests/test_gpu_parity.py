@@ -380,6 +380,39 @@ def test_sparse_attn_with_token_mask(cfg, n_text, kind):
     plan.close()
 
 
+@pytest.mark.parametrize("cfg,n_text", [(CFG_TINY, 0), (CFG_RAGGED64, 0), (CFG_RAGGED128, 0), (CFG_MID128, 0),
+                                        (CFG_RAGGED64, 50), (CFG_MID128, 100)],
+                         ids=["tiny", "ragged64", "ragged128", "mid128", "ragged64+text", "mid128+text"])
+@pytest.mark.parametrize("kind", ["entropy", "small", "uniform"])
+def test_sparse_attn_token_level_without_block_list(cfg, n_text, kind):
+    """ridx and no block list: Eq. 16 itself (oracle mode 2) — every query over exactly the keys inside
+    its disk; the kernel derives the reachable key blocks from the plan's boxes."""
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg, n_text=n_text)
+    S, b = geo.N + n_text, geo.block
+    Qr, Kr, Vr = workloads.make_qkv(cfg, DEV)
+    if n_text:
+        Qr, Kr, Vr = workloads.append_text(Qr, Kr, Vr, cfg, n_text)
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    rv = random_ridx(geo, cfg["heads"], np.random.default_rng(41), kind)
+    ridx = np.full((cfg["heads"], S), geo.radii.size - 1, np.uint16)
+    ridx[:, : geo.N] = rv
+    ridx_t = torch.from_numpy(ridx.view(np.int16)).to(DEV)[None]
+    O, lse = plan.sparse_attn(Q, K, V, None, None, ridx=ridx_t, want_lse=True)
+    plan.check_status()
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(S)
+    for h in range(cfg["heads"]):
+        vis2 = oracle.visible_rows(geo.coord, geo.T, b, geo.theta, ridx[h], rows, None, 2, n_text=n_text)
+        assert vis2.any(axis=1).all()              # a query always sees itself
+        ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis2)
+        common.assert_output(O[0, h], ref["O"], f"token-level head {h}")
+        assert np.abs(lse[0, h].cpu().numpy().astype(np.float64) - ref["lse"]).max() <= 4e-3
+    with pytest.raises(api().TraError):
+        plan.sparse_attn(Q, K, V, None, None)       # neither a block list nor radii
+    plan.close()
+
+
 def test_sparse_attn_full_mask_equals_dense():
     # every block retained: the sparse call reproduces dense attention (full-support radius)
     cfg = CFG_RAGGED128
@@ -456,6 +489,7 @@ def test_full_size_sampled_rows(name, heads_checked, n_random):
     mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
     Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
     Ot, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx)      # token mask inside the blocks
+    Oe, _ = plan.sparse_attn(Q, K, V, None, None, ridx=ridx)            # Eq. 16 itself, no block list
     plan.check_status()
     rng = np.random.default_rng(15)
     for h in heads_checked:
@@ -486,6 +520,9 @@ def test_full_size_sampled_rows(name, heads_checked, n_random):
         assert vis1.sum() < vis.sum()
         reft = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis1)
         common.assert_output(Ot[0, h][rows_t], reft["O"], f"token mask {name} h{h}")
+        vis2 = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_np, rows, None, 2)
+        refe = oracle.attention_rows(Qb, Kb, Vb, common.scale_of(cfg), rows, vis2)
+        common.assert_output(Oe[0, h][rows_t], refe["O"], f"token level {name} h{h}")
     # CSR of every head is the ascending list of the mask the same call wrote
     m = mask[0].reshape(-1, geo.NB).bool()
     counts = m.sum(dim=1)
