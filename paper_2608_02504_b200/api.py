@@ -300,7 +300,19 @@ class HostPipeline:
         self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.dev)
         self._ws_ptr = (self.workspace.data_ptr() + 255) & ~255
         self.launches_per_group = 10      # 3 gathers, dense, budget, vote + scan + fill, sparse, scatter
-        self.n_groups = 1 + -(-(heads - self.first_group) // self.group)
+        self.n_groups = len(self.group_sizes(heads, self.group, self.first_group))
+
+    @staticmethod
+    def group_sizes(heads, group, first_group):
+        """The head groups of one pass (mirrors the library): a small first and a small last group."""
+        sizes, left = [], heads
+        while left > 0:
+            n = min(first_group if not sizes else group, left)
+            if left - n == 0 and n > first_group and sizes:
+                n -= first_group
+            sizes.append(n)
+            left -= n
+        return sizes
 
     @staticmethod
     def _check_host(t, shape, name):

@@ -98,9 +98,18 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
 
   cudaEvent_t in_free[2] = {nullptr, nullptr};    // the gathers that read staging buffer b are done
   cudaEvent_t out_free[2] = {nullptr, nullptr};   // the copy out of output buffer b is done
+  // group sizes: a small first group (the kernels start early) and a small last one (little output
+  // left to copy after the last kernel)
+  std::vector<int> sizes;
+  for (int left = heads; left > 0;) {
+    int n = std::min(sizes.empty() ? first_group : group, left);
+    if (left - n == 0 && n > first_group && !sizes.empty()) n -= first_group;   // split the last group
+    sizes.push_back(n);
+    left -= n;
+  }
   int h0 = 0;
-  for (int i = 0; h0 < heads; ++i) {
-    const int n = std::min(i == 0 ? first_group : group, heads - h0);
+  for (int i = 0; i < (int)sizes.size(); ++i) {
+    const int n = sizes[i];
     const int b = i & 1;
     // inputs of this group: host -> staging buffer b
     if (in_free[b]) TRA_CUDA_CHECK(cudaStreamWaitEvent(s_in, in_free[b], 0));

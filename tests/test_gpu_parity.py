@@ -689,8 +689,9 @@ def test_host_pipeline_matches_device_path():
             launches = pipe.run(host[0], host[1], host[2], out)
             torch.cuda.synchronize()
             assert torch.equal(out, expect)
-        n_groups = -(-cfg["heads"] // min(group, cfg["heads"])) if first is None else 1 + -(-(cfg["heads"] - first) // group)
-        assert launches == 10 * n_groups
+        sizes = api().HostPipeline.group_sizes(cfg["heads"], pipe.group, pipe.first_group)
+        assert sum(sizes) == cfg["heads"] and max(sizes) <= pipe.group and sizes[0] <= pipe.first_group
+        assert launches == 10 * len(sizes)
     with pytest.raises(ValueError):
         pipe.run(Qr, host[1], host[2], out)     # a device tensor where a pinned host tensor belongs
     # the C entry point refuses a workspace that is too small or misaligned, before any work
