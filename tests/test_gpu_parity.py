@@ -475,7 +475,8 @@ def sampled_rows(geo, rng, n_random):
 
 
 @pytest.mark.parametrize("name,heads_checked,n_random",
-                         [("wan1.3b-480p", (0, 11), 26), ("wan14b-720p", (0, 39), 22), ("hunyuan-720p", (0, 23), 14)])
+                         [("wan1.3b-480p", (0, 3, 7, 11), 100), ("wan14b-720p", (0, 13, 26, 39), 100),
+                          ("hunyuan-720p", (0, 7, 15, 23), 60)])
 def test_full_size_sampled_rows(name, heads_checked, n_random):
     """At the BASELINE shapes, all heads resident, in the launch configuration the benchmark times:
     sampled (head, row) pairs of dense attention + entropy, the integer stages of their block
