@@ -390,6 +390,12 @@ def run_ours(args):
         K.copy_(k_keep)
         del q_keep, k_keep
 
+    # ---- tile-shape sweep of the tile-major order (the paper's tile-size ablation) ----------------
+    tile_sweep = None
+    if args.tile_sweep and rank == 0:
+        tile_sweep = [run_tile_shape(api, cfg, th, tw, Qr, Kr, Vr, dev)
+                      for th, tw in ((8, 16), (16, 8), (4, 32), (1, cfg["W"]))]
+
     # ---- the other shapes the paper measures on (same pass, stage times only) ------------------
     other = None
     if args.other_workloads and rank == 0 and args.config == "wan14b-720p" and args.heads is None:
@@ -418,7 +424,7 @@ def run_ours(args):
                        "l2": "inputs larger than L2 (Q/K/V/O are 774 MB each)"},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "roofline_sparse": roofline_sparse, "stages": stages,
-            "tau_sweep": tau_sweep, "other_workloads": other, "schedule": schedule, "cpu_baseline": cpu_baseline,
+            "tau_sweep": tau_sweep, "tile_sweep": tile_sweep, "other_workloads": other, "schedule": schedule, "cpu_baseline": cpu_baseline,
             "paper_context": "paper: 1.56-2.05x end-to-end speedup at 9-19% retained interactions on one H200",
             "wall_s_timed_region": round(wall_s, 3),
         }
@@ -482,6 +488,34 @@ def run_schedule(cfg, plan, api, dev, bufs, n_steps, n_warm, refresh_every=0, en
             "sparse_step_ms": round(float(np.mean(per_step[n_warm:])), 3),
             "retained_block_density": round(computed_pairs(mask, N, block) / (heads * float(N) * N), 4),
             "drift": "Q and K: x_t = x_{t-1} + 0.05 N(0,1) on the fp32 state; V fixed"}
+
+
+def run_tile_shape(api, cfg, tile_h, tile_w, Qr, Kr, Vr, dev):
+    """The same layer with another tile shape of the tile-major order (blocks stay `block` consecutive
+    positions): retained density and sparse time.  One warm-up pass, one timed sparse launch pair."""
+    c = dict(cfg, tile_h=tile_h, tile_w=tile_w)
+    N, heads, block = workloads.num_tokens(c), c["heads"], c["block"]
+    plan = api.Plan.from_config(c)
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    O, H, _ = plan.entropy_attn(Q, K, V)
+    _, _, ridx = plan.budget_radius(H, want_budget=False, want_radius=False)
+    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
+    plan.sparse_attn(Q, K, V, row_ptr, col_idx, O=O)
+    torch.cuda.synchronize()
+    e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    e0.record()
+    plan.build_block_mask(ridx, mask, row_ptr, col_idx, nnz)
+    e1.record()
+    for _ in range(2):
+        plan.sparse_attn(Q, K, V, row_ptr, col_idx, O=O)
+    e2.record()
+    torch.cuda.synchronize()
+    plan.check_status()
+    out = {"tile": [tile_h, tile_w],
+           "block_density": round(computed_pairs(mask, N, block) / (heads * float(N) * N), 4),
+           "sparse_ms": round(e1.elapsed_time(e2) / 2, 3), "block_mask_ms": round(e0.elapsed_time(e1), 3)}
+    plan.close()
+    return out
 
 
 def run_other_workload(api, name, dev, peak_tf, reps=2):
@@ -661,6 +695,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-schedule", dest="schedule", action="store_false")
     ap.add_argument("--no-tau-sweep", dest="tau_sweep", action="store_false")
+    ap.add_argument("--no-tile-sweep", dest="tile_sweep", action="store_false",
+                    help="skip the tile-shape sweep of the tile-major order")
     ap.add_argument("--no-other-workloads", dest="other_workloads", action="store_false",
                     help="skip the Wan2.1-1.3B and HunyuanVideo shapes reported next to the main workload")
     args = ap.parse_args()
