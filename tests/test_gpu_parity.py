@@ -28,8 +28,10 @@ CFG_RAGGED64 = common.small_config(3, 7, 10, heads=3, head_dim=64, block=64, til
 CFG_RAGGED128 = common.small_config(5, 9, 11, heads=2, head_dim=128, block=128, tile_h=4, tile_w=4, seed=79)
 CFG_MID128 = common.small_config(6, 16, 24, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16, seed=80,
                                  s_lo=0.2, s_hi=5.0)
-SMALL = [CFG_TINY, CFG_RAGGED64, CFG_RAGGED128, CFG_MID128]
-IDS = ["tiny", "ragged64", "ragged128", "mid128"]
+# head_dim 128 with 64-token blocks (two query blocks per 128-row tile), ragged: N = 378
+CFG_D128_B64 = common.small_config(3, 9, 14, heads=2, head_dim=128, block=64, tile_h=4, tile_w=8, seed=81)
+SMALL = [CFG_TINY, CFG_RAGGED64, CFG_RAGGED128, CFG_MID128, CFG_D128_B64]
+IDS = ["tiny", "ragged64", "ragged128", "mid128", "d128b64"]
 
 
 def make_plan(cfg, **kw):
