@@ -174,13 +174,13 @@ def _random_geometries(n, seed):
         block = int(rng.choice([64, 128]))
         th, tw = int(rng.choice([1, 2, 4, 8, 16])), int(rng.choice([4, 8, 16, 32]))
         out.append(common.small_config(int(rng.integers(1, 7)), int(rng.integers(3, 34)), int(rng.integers(3, 50)),
-                                       heads=2, head_dim=64, block=block, tile_h=th, tile_w=tw,
+                                       heads=2, head_dim=int(rng.choice([64, 128])), block=block, tile_h=th, tile_w=tw,
                                        gamma=float(rng.choice([0.0, 0.0513, 0.6, 0.95, 2.0])),
                                        tau=float(rng.choice([0.3, 0.5, 0.9, 1.0])), seed=200 + i))
     return out
 
 
-@pytest.mark.parametrize("cfg", _random_geometries(10, 5), ids=lambda c: f"{c['T']}x{c['H']}x{c['W']}-b{c['block']}-"
+@pytest.mark.parametrize("cfg", _random_geometries(10, 5), ids=lambda c: f"{c['T']}x{c['H']}x{c['W']}-d{c['head_dim']}-b{c['block']}-"
                                                                          f"t{c['tile_h']}x{c['tile_w']}")
 def test_random_geometries_integer_stages_and_token_mask(cfg):
     """Seeded random grids, tile shapes, decay rates and target masses: plan tables, budget, radius,
@@ -211,13 +211,21 @@ def test_random_geometries_integer_stages_and_token_mask(cfg):
     assert int(nnz.item()) == rp[-1]
     assert np.array_equal(row_ptr.cpu().numpy().astype(np.int64), rp)
     assert np.array_equal(col_idx.cpu().numpy()[: rp[-1]], ci)
-    # token mask inside the retained blocks
+    # dense attention + entropy, block-sparse attention, and the token mask inside the retained blocks
     Q, K, V = tile_major_inputs(cfg, plan)
+    Od, Hd, _ = plan.entropy_attn(Q, K, V)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
     O, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx_t)
     plan.check_status()
     Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
     rows = np.arange(geo.N)
     for h in range(heads):
+        rd = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows)
+        common.assert_output(Od[0, h], rd["O"], f"dense head {h}")
+        assert np.abs(Hd[0, h].cpu().numpy() - rd["H_def"]).max() <= common.ENTROPY_ATOL
+        vis0 = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_ref[h], rows, ref[h][rows // geo.block], 0)
+        rs = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis0)
+        common.assert_output(Os[0, h], rs["O"], f"sparse head {h}")
         vis1 = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx_ref[h], rows, ref[h][rows // geo.block], 1)
         r = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis1)
         common.assert_output(O[0, h], r["O"], f"token-mask head {h}")
