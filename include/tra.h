@@ -127,9 +127,8 @@ int tra_tile_major_scatter(const tra_plan_t* plan, const void* src_tile_major, v
  *   Q, K, V : bf16 [B, heads, N, head_dim], 128-byte aligned.
  *   O       : bf16, same shape (written).
  *   entropy : fp32 [B, heads, N] or NULL (NULL = plain dense attention, no entropy work).
- *   lse     : fp32 [B, heads, N] or NULL; log sum_j exp(s_ij).  Exact to fp32 rounding when
- *             entropy is requested; otherwise formed from the bf16-rounded probabilities
- *             (absolute error up to about 4e-3).
+ *   lse     : fp32 [B, heads, N] or NULL; log sum_j exp(s_ij), exact to fp32 rounding (the row sum
+ *             of the unrounded probabilities is kept next to the bf16-rounded one that normalises O).
  *   sm_scale: multiplies q.k; pass 1/sqrt(head_dim) for Eq. 1. */
 int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O,
                      float* entropy, float* lse, int B, int heads, float sm_scale, void* stream);
@@ -150,12 +149,19 @@ int tra_budget_radius(const tra_plan_t* plan, const float* entropy, int32_t* bud
  *   ridx      : uint16 [B, heads, N] from tra_budget_radius.
  *   block_mask: uint8 [B, heads, NB, NB] (written, 0/1).
  *   row_ptr   : int32 [B*heads*NB + 1] (written); col_idx: int32 [col_idx_capacity] (written,
- *               ascending inside a row).  If nnz exceeds the capacity, col_idx is left partly
- *               written and TRA_ERR_CAPACITY is recorded in the plan status.
- *   nnz_out   : device int64 or NULL; total retained blocks. */
+ *               ascending inside a row).  If nnz exceeds the capacity, TRA_ERR_CAPACITY is recorded
+ *               in the plan status, col_idx holds the first `capacity` entries and every row_ptr
+ *               offset is clamped to the capacity, so that a later tra_sparse_attn stays inside
+ *               col_idx (its result is then incomplete; read the status).
+ *   nnz_out   : device int64 or NULL; total retained blocks.
+ *   tile_pairs: int32 [B*heads, ceil(NT/2), 2] or NULL, NT = ceil(S / 128) (written).  The paper has
+ *               no counterpart: tra_sparse_attn gives each thread block two 128-row query tiles that
+ *               share the key/value tiles they both retain, and this table pairs tiles whose block
+ *               lists are similar (entry -1 = no second tile).  Pass it to tra_sparse_attn together
+ *               with row_ptr / col_idx; it changes the speed of that call, never its result. */
 int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* block_mask,
                          int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
-                         int64_t* nnz_out, int B, int heads, void* stream);
+                         int64_t* nnz_out, int32_t* tile_pairs, int B, int heads, void* stream);
 
 /* Block-sparse attention (Eq. 16 as executed: Section 3.2, last paragraph, and "Limitations"):
  * softmax attention of each query over the valid keys of the retained key blocks of its block row.
@@ -170,11 +176,14 @@ int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* 
  *                 from the plan's block boxes; no [heads, NB, NB] mask is needed.
  * A query that is left with no visible key gets O = 0 and lse = -inf.
  *   row_ptr, col_idx: the CSR list written by tra_build_block_mask (reusable across calls:
- *   Section 3.3, warm-up reuse).  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL; formed
- *   from the bf16-rounded probabilities (absolute error up to about 4e-3). */
+ *   Section 3.3, warm-up reuse).  tile_pairs: the table the same call wrote, or NULL (consecutive
+ *   tiles share a thread block); any table in which every tile 0 .. NT-1 of a (batch, head) appears
+ *   exactly once gives the same result.  Q, K, V, O as in tra_entropy_attn.  lse: fp32 or NULL, exact
+ *   to fp32 rounding. */
 int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
-                    const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, void* O,
-                    float* lse, int B, int heads, float sm_scale, void* stream);
+                    const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx,
+                    const int32_t* tile_pairs, void* O, float* lse, int B, int heads, float sm_scale,
+                    void* stream);
 
 /* ---- the whole pass over HOST tensors (the paper has no counterpart: plumbing around the calls
  * above for callers whose Q, K, V and O live in host memory) ----------------------------- */

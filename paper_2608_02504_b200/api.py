@@ -13,7 +13,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libtra_b200.so")
+# TRA_B200_LIB selects another build of the same library (the bounds-checking debug build)
+LIB_PATH = os.environ.get("TRA_B200_LIB") or os.path.join(_HERE, "libtra_b200.so")
 
 TRA_OK = 0
 TRA_KEEP_DIAGONAL = 1
@@ -67,8 +68,8 @@ def _load():
     lib.tra_tile_major_scatter.argtypes = [vp, vp, vp, i32, i32, vp]
     lib.tra_entropy_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
     lib.tra_budget_radius.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
-    lib.tra_build_block_mask.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int64, vp, i32, i32, vp]
-    lib.tra_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
+    lib.tra_build_block_mask.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int64, vp, vp, i32, i32, vp]
+    lib.tra_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
     return lib
 
 
@@ -234,8 +235,16 @@ class Plan:
                "tra_budget_radius")
         return budget, radius, ridx
 
-    def build_block_mask(self, ridx, block_mask=None, row_ptr=None, col_idx=None, nnz=None):
-        """ridx [B, heads, N] -> (block_mask uint8 [B, heads, NB, NB], row_ptr, col_idx, nnz)."""
+    @property
+    def n_tile_pairs(self):
+        """Thread blocks per (batch, head) of a block-sparse launch: pairs of 128-row query tiles."""
+        return ((self.N + 127) // 128 + 1) // 2
+
+    def build_block_mask(self, ridx, block_mask=None, row_ptr=None, col_idx=None, nnz=None, tile_pairs=None,
+                         want_tile_pairs=False):
+        """ridx [B, heads, N] -> (block_mask uint8 [B, heads, NB, NB], row_ptr, col_idx, nnz); with
+        ``want_tile_pairs`` (or a ``tile_pairs`` buffer) a fifth result: the int32 [B*heads, pairs, 2]
+        table of query tiles that share a thread block in ``sparse_attn``."""
         B, heads = ridx.shape[0], ridx.shape[1]
         dev = ridx.device
         rows = B * heads * self.NB
@@ -247,16 +256,21 @@ class Plan:
             col_idx = torch.empty(rows * self.NB, dtype=torch.int32, device=dev)
         if nnz is None:
             nnz = torch.zeros(1, dtype=torch.int64, device=dev)
+        if tile_pairs is None and want_tile_pairs:
+            tile_pairs = torch.empty(B * heads, self.n_tile_pairs, 2, dtype=torch.int32, device=dev)
         _check(_lib.tra_build_block_mask(self._h, _dev(ridx, torch.int16, "ridx"),
                                          _dev(block_mask, torch.uint8, "block_mask"),
                                          _dev(row_ptr, torch.int32, "row_ptr"),
                                          _dev(col_idx, torch.int32, "col_idx"), col_idx.numel(),
-                                         _dev(nnz, torch.int64, "nnz"), B, heads, _stream()),
+                                         _dev(nnz, torch.int64, "nnz"), _dev(tile_pairs, torch.int32, "tile_pairs"),
+                                         B, heads, _stream()),
                "tra_build_block_mask")
+        if tile_pairs is not None:
+            return block_mask, row_ptr, col_idx, nnz, tile_pairs
         return block_mask, row_ptr, col_idx, nnz
 
     def sparse_attn(self, Q, K, V, row_ptr, col_idx, O=None, lse=None, want_lse=False, sm_scale=None,
-                    ridx=None):
+                    ridx=None, tile_pairs=None):
         """Block-sparse attention over the retained key blocks (tile-major inputs).  With ``ridx`` the
         token mask of Eq. 15 is applied inside the retained blocks as well; with ``ridx`` and
         ``row_ptr = col_idx = None`` the call evaluates Eq. 16 itself (token mask alone, no block list)."""
@@ -270,7 +284,7 @@ class Plan:
         _check(_lib.tra_sparse_attn(self._h, _dev(Q, bf, "Q"), _dev(K, bf, "K"), _dev(V, bf, "V"),
                                     _dev(row_ptr, torch.int32, "row_ptr"),
                                     _dev(col_idx, torch.int32, "col_idx"), _dev(ridx, torch.int16, "ridx"),
-                                    _dev(O, bf, "O"),
+                                    _dev(tile_pairs, torch.int32, "tile_pairs"), _dev(O, bf, "O"),
                                     _dev(lse, torch.float32, "lse"), B, heads, scale, _stream()),
                "tra_sparse_attn")
         return O, lse
@@ -299,7 +313,7 @@ class HostPipeline:
         self.workspace_bytes = int(_lib.tra_hot_path_host_workspace_bytes(plan._h, self.group))
         self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.dev)
         self._ws_ptr = (self.workspace.data_ptr() + 255) & ~255
-        self.launches_per_group = 10      # 3 gathers, dense, budget, vote + scan + fill, sparse, scatter
+        self.launches_per_group = 11      # 3 gathers, dense, budget, vote + scan + fill + pairing, sparse, scatter
         self.n_groups = len(self.group_sizes(heads, self.group, self.first_group))
 
     @staticmethod

@@ -1,992 +1,26 @@
-// Dense attention with fused entropy (Eq. 1, Eq. 2, Algorithm 2) and block-sparse attention
-// (Eq. 16 as executed over retained blocks) for sm_100a.
-//
-// One CTA owns 256 consecutive query positions of one (batch, head): two 128-row query tiles.
-// Both S = Q K^T and O += P V run on the 5th-generation tensor cores (tcgen05.mma, kind::f16,
-// bf16 operands, fp32 accumulators in tensor memory).  K/V tiles of the retained key blocks are
-// fetched by TMA into a shared-memory ring.  Warp roles:
-//   warps 0-3  softmax of query tile 0 (one thread per query row, tcgen05.ld of its S row)
-//   warps 4-7  softmax of query tile 1
-//   warp  8    TMA producer (Q once, then K_v, V_v for every key block v of the CTA's list)
-//   warp  9    tensor-memory allocation and the single MMA-issuing thread
-//   warps 10-11 idle: they complete the third warpgroup, whose registers are handed to the softmax
-//              warps with setmaxnreg so that a softmax thread can keep its whole S row in registers
-// Tensor-memory columns: S0 [0,128)  S1 [128,256)  O0 [256,384)  O1 [384,512); the bf16 P of a
-// tile overwrites the first half of its S columns and feeds the PV MMA straight from tensor memory.
-// The two tiles alternate on the tensor pipe (PV_k(e) then S_k(e+1)) while the other tile's
-// softmax runs.  The key-block list of the CTA is the union of the lists of the query blocks it
-// holds; a tile skips the MMAs of a key block none of its query blocks retains.  Dense launches
-// (kDense) have no list and count key blocks instead.  With kTokenMask the softmax threads also
-// remove, inside every retained block, the keys outside their query's disk (Eq. 15).
-//
-// Online softmax state per row, in the base-2 domain (t = s * sm_scale * log2 e):
-//   m  running reference maximum (raised only when the new maximum exceeds it by more than 8,
-//      so the O accumulator is rescaled rarely; exact because every term uses the same m),
-//   l  = sum 2^(t - m),   a = sum 2^(t - m) (t - m)   (the entropy accumulator of Algorithm 2,
-//      centred on m, which keeps its magnitude small).
-// At the end  O = o / l,  lse = (m + log2 l) ln 2,  H = ln l - ln 2 * a / l
-// (= m + log l - (sum e^(s-m) s) / l of Algorithm 2 with s measured from m).
-//
-// Every wait on an mbarrier is bounded: after about two seconds the waiting thread records
-// TRA_ERR_TIMEOUT in the plan's status word, raises a CTA-wide abort flag and every role leaves
-// its loop; tensor memory is released on every path.
-#include <cuda.h>
-#include <cuda_bf16.h>
-
-#include "tra_common.cuh"
+// Entry points of the attention calls: argument checks, shape dispatch, and the self-test of the
+// bounded device-side wait.  The kernels live in tra_attn_kernel.cuh, one translation unit per shape.
+#include "tra_attn_kernel.cuh"
 
 namespace {
 
-constexpr int kThreads = 384;         // 12 warps: three per SM sub-partition
-constexpr int kRegsSoftmax = 216;     // per-thread registers after setmaxnreg: 2 * 216 + 72 = 3 * 168
-constexpr int kRegsControl = 72;
-constexpr int kTileM = 128;           // query rows per tile (UMMA M)
-constexpr int kMaxBitmapWords = 64;   // key blocks per row <= 2048
-constexpr float kLog2e = 1.4426950408889634f;
-constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kRescaleThreshold = 8.0f;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
-
-// ------------------------------------------------------------------------------------ PTX
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.b32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait; false = gave up (abort flag raised by this or another thread).
-__device__ __forceinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                            int* status, unsigned long long limit_ns = kWaitLimitNs) {
-  // The global timer is slow to read, so it is consulted only after many failed polls (each
-  // try_wait already suspends the thread for a while): ordinary waits never touch it.
-#pragma unroll 1
-  for (uint32_t it = 0; it < 4096u; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if (globaltimer_ns() - t0 > limit_ns) {
-        *abort_flag = 1;
-        tra_set_status(status, TRA_ERR_TIMEOUT);
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status);
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
-                                            int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, "
-      "%4}], [%5];" ::"r"(dst),
-      "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-      : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() {
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_after() {
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-// The MMA warp runs its loop with all 32 lanes (warp-uniform control flow and descriptor
-// arithmetic); the tcgen05.mma / tcgen05.commit instructions themselves are issued by one elected lane.
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile(
-      "{\n\t.reg .pred pe;\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
-      "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar)
-      : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem].  Descriptors arrive as (lo, hi) words so that stepping along K
-// is one 32-bit add on the issuing thread.
-__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
-                                          uint32_t b_hi, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, pe;\n\t.reg .b64 da, db;\n\t"
-      "mov.b64 da, {%1, %2};\n\t"
-      "mov.b64 db, {%3, %4};\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
-      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
-                                          uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p, pe;\n\t.reg .b64 db;\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "elect.sync _|pe, 0xffffffff;\n\t"
-      "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(d_tmem),
-      "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-
-// 32 consecutive fp32 columns of this thread's tensor-memory lane
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]),
-      "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]),
-      "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-      "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-      : "memory");
-}
-// Waits for this thread's tcgen05.ld; the 32 destination registers are named as read-write
-// operands so that the compiler cannot move a use of them above the wait.
-__device__ __forceinline__ void tmem_wait_ld(uint32_t* r) {
-  asm volatile("tcgen05.wait::ld.sync.aligned;"
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
-                 "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
-                 "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
-                 "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
-                 "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :
-               : "memory");
-}
-// Compiler-only fence on 32 registers filled by an earlier tcgen05.ld: keeps their uses below
-// the tcgen05.wait::ld that precedes this statement.
-__device__ __forceinline__ void reg_fence32(uint32_t* r) {
-  asm volatile(""
-               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]),
-                 "+r"(r[7]), "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]),
-                 "+r"(r[14]), "+r"(r[15]), "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]),
-                 "+r"(r[21]), "+r"(r[22]), "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]),
-                 "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-               :
-               : "memory");
-}
-__device__ __forceinline__ void tmem_wait_st() {
-  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ float ex2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float fmax3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-// ---- packed fp32 pairs (sm_100 f32x2 arithmetic: one instruction for two lanes of a row) ----
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t fadd2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-// floor(sqrt(n)) for 0 <= n < 2^22 with no conversion instruction (conversions share the
-// special-function unit with ex2): n + 0.5 is formed from the 2^23 bit pattern, sqrt.approx of it
-// stays at least 0.25 / sqrt(n) away from every integer, and adding 2^23 - 0.5 rounds it down into
-// the low mantissa bits.
-__device__ __forceinline__ int tra_isqrt_small_nocvt(int n) {
-  const float f = __uint_as_float(0x4B000000u | (uint32_t)n) - 8388607.5f;      // n + 0.5, exact
-  float r;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(f));
-  return (int)(__float_as_uint(r + 8388607.5f) & 0x7FFFFFu);
-}
-// bf16x2 with `lo` in the low half
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-  uint32_t d;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-  return d;
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle, sm_100 format (version 1), as two words:
-//   lo = start address >> 4 (14 bits) | leading byte offset >> 4 at bit 16
-//   hi = stride byte offset >> 4 | version 1 at bit 14 | SWIZZLE_128B (2) at bits 29..31
-__device__ __forceinline__ uint32_t desc_lo(uint32_t saddr, uint32_t lbo_bytes) {
-  return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
-}
-__host__ __device__ constexpr uint32_t desc_hi(uint32_t sbo_bytes) {
-  return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (2u << 29);
-}
-
-// Instruction descriptor, kind::f16: fp32 accumulate, bf16 x bf16, M = 128.
-__host__ __device__ constexpr uint32_t make_idesc(int n, bool b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
-         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
-}
-
-template <int D, int BN>
-struct Cfg {
-  static constexpr int kGroups = kTileM / BN;                 // query blocks per tile
-  static constexpr int kBlocksPerCta = 2 * kGroups;
-  static constexpr int kQTileBytes = kTileM * D * 2;
-  static constexpr int kSlotBytes = BN * D * 2;
-  static constexpr int kSlots = (D == 128 && BN == 128) ? 5 : 6;
-  static constexpr int kAtoms = D / 64;                        // 64-column swizzle atoms per row
-  static constexpr int kQAtomBytes = kTileM * 128;
-  static constexpr int kKVAtomBytes = BN * 128;
-  static constexpr int kSmemData = 2 * kQTileBytes + kSlots * kSlotBytes;
-  // at least 120 KB so that one CTA owns an SM and its whole tensor memory
-  static constexpr int kSmemNeeded = kSmemData + 1024 /*alignment slack*/ + 2048 /*barriers, bitmaps*/;
-  static constexpr int kSmemBytes = kSmemNeeded > 120 * 1024 ? kSmemNeeded : 120 * 1024;
-};
-
-struct SharedCtl {
-  uint64_t q_full;
-  uint64_t kv_full[6];
-  uint64_t kv_release[4];   // ring slots are handed back in release events (see the MMA warp)
-  uint64_t s_full[2];
-  uint64_t p_ready[2][2];   // [tile][64-key half of the block]
-  uint64_t drain;
-  uint32_t tmem_base;
-  int abort_flag;
-  int rmax[4];              // largest candidate index among the video queries of each query block
-  uint32_t bitmap[4][kMaxBitmapWords];
-};
-static_assert(sizeof(SharedCtl) <= 2048, "control block");
-
-// Arguments of the optional token mask inside retained blocks (Eq. 15 applied on top of the block
-// list): packed coordinates of the video tokens (padded by one block), thresholds, candidate indices.
-struct TokenMaskArgs {
-  const tra_block_boxes_t* boxes; // per-block boxes (plan table), for launches without a block list
-  const uint32_t* slice;          // one word per 16 positions (plan table): run of one frame row or 0
-  const uint32_t* coord_packed;
-  const int32_t* theta;
-  const uint16_t* ridx;
-  int n_video;
-  int T;
-};
-
-// ------------------------------------------------------------------------------------ kernel
-// kDense: every query block attends to every key block (no block list; row_ptr is not read).
-template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense>
-__global__ void __launch_bounds__(kThreads, 1)
-tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ O,
-                float* __restrict__ entropy, float* __restrict__ lse,
-                const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx, int N, int NB,
-                float scale_log2, int* __restrict__ status, TokenMaskArgs tm) {
-  using C = Cfg<D, BN>;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;                                   // [2 tiles][atoms][128 rows][64] bf16, swizzled
-  uint8_t* sKV = smem + 2 * C::kQTileBytes;             // ring of K / V tiles
-  SharedCtl* ctl = (SharedCtl*)(smem + C::kSmemData);
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int pair = blockIdx.x;
-  const int bh = blockIdx.y;
-  const int q_base = pair * 2 * kTileM;
-  const int n_words = (NB + 31) >> 5;
-  volatile int* abort_flag = &ctl->abort_flag;
-
-  // ---- set-up --------------------------------------------------------------------------
-  if (tid == 0) {
-    mbar_init(smem_u32(&ctl->q_full), 1);
-    for (int i = 0; i < C::kSlots; ++i) {
-      mbar_init(smem_u32(&ctl->kv_full[i]), 1);
-    }
-    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&ctl->kv_release[i]), 1);
-    for (int k = 0; k < 2; ++k) {
-      mbar_init(smem_u32(&ctl->s_full[k]), 1);
-      mbar_init(smem_u32(&ctl->p_ready[k][0]), 4);     // one lane of each of the tile's four warps
-      mbar_init(smem_u32(&ctl->p_ready[k][1]), 4);
-    }
-    mbar_init(smem_u32(&ctl->drain), 1);
-    ctl->abort_flag = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
-  if (warp == 9) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(
-                     smem_u32(&ctl->tmem_base))
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  for (int i = tid; i < 4 * kMaxBitmapWords; i += kThreads) (&ctl->bitmap[0][0])[i] = 0u;
-  if (tid < 4) ctl->rmax[tid] = -1;
-  __syncthreads();
-  // Token-mask launch without a block list (Eq. 16 itself): the key blocks a query block can reach
-  // at all, from the block boxes and the largest candidate index among its queries — a superset
-  // of the blocks that hold a visible key; the token mask inside the kernel does the rest.
-  const bool geometric_list = kTokenMask && row_ptr == nullptr;
-  if (geometric_list) {
-    for (int i = tid; i < 2 * kTileM; i += kThreads) {
-      const int row = q_base + i;
-      if (row < tm.n_video) atomicMax(&ctl->rmax[i / BN], (int)tm.ridx[(size_t)bh * N + row]);
-    }
-    __syncthreads();
-    for (int g = 0; g < C::kBlocksPerCta; ++g) {
-      const int ub = pair * C::kBlocksPerCta + g;
-      if (ub >= NB) continue;
-      const bool q_text = (ub + 1) * BN > tm.n_video;        // holds a text query: sees every key
-      const int rmax = ctl->rmax[g];
-      const tra_block_boxes_t ubx = tm.boxes[ub];
-      for (int v = tid; v < NB; v += kThreads) {
-        bool on = q_text || (v + 1) * BN > tm.n_video;         // text keys are always visible
-        if (!on && rmax >= 0) {
-          const tra_block_boxes_t vb = tm.boxes[v];
-          for (int iu = 0; iu < ubx.n_box && !on; ++iu)
-            for (int iv = 0; iv < vb.n_box && !on; ++iv) {
-              const tra_box_t a = ubx.box[iu], c = vb.box[iv];
-              const int dt_min = max(0, max(a.t0 - c.t1, c.t0 - a.t1));
-              const int gy = max(0, max(a.y0 - c.y1, c.y0 - a.y1));
-              const int gx = max(0, max(a.x0 - c.x1, c.x0 - a.x1));
-              on = tm.theta[rmax * tm.T + dt_min] >= gy * gy + gx * gx;
-            }
-        }
-        if (on) atomicOr(&ctl->bitmap[g][v >> 5], 1u << (v & 31));
-      }
-    }
-  }
-  // key-block bitmaps of the query blocks this CTA holds (block-sparse launches only)
-  for (int g = 0; g < C::kBlocksPerCta && !kDense && !geometric_list; ++g) {
-    const int ub = pair * C::kBlocksPerCta + g;
-    if (ub >= NB) continue;
-    {
-      const long long r = (long long)bh * NB + ub;
-      const int lo = row_ptr[r], hi = row_ptr[r + 1];
-      for (int e = lo + tid; e < hi; e += kThreads) {
-        const int v = col_idx[e];
-        if (v >= 0 && v < NB) atomicOr(&ctl->bitmap[g][v >> 5], 1u << (v & 31));
-      }
-    }
-  }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem = ctl->tmem_base;
-
-  // dense launches: a tile takes part when its first query block exists
-  const bool tile1_on = pair * C::kBlocksPerCta + C::kGroups < NB;
-  const int n_outer = kDense ? 1 : n_words;   // dense launches walk 0 .. NB-1 in one inner loop
-  // bitmap of a tile = union over its query blocks
-  auto tile_word = [&](int k, int w) -> uint32_t {
-    uint32_t x = ctl->bitmap[k * C::kGroups][w];
-    if (C::kGroups == 2) x |= ctl->bitmap[k * C::kGroups + 1][w];
-    return x;
-  };
-
-  if (warp >= 8) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsControl));
-  if (warp == 8) {
-    // ================================================================== TMA producer
-    if (lane == 0) {
-      const uint32_t qbar = smem_u32(&ctl->q_full);
-      mbar_expect_tx(qbar, 2 * C::kQTileBytes);
-      for (int k = 0; k < 2; ++k)
-        for (int a = 0; a < C::kAtoms; ++a)
-          tma_load_3d(smem_u32(sQ + k * C::kQTileBytes + a * C::kQAtomBytes), &map_q, qbar, a * 64,
-                      q_base + k * kTileM, bh);
-      int slot = 0;
-      bool alive = true;
-      // Loads go K0, V0, K1, V1, ... into consecutive slots.  The MMA warp hands slots back in
-      // release events: event 0 frees K0, event e + 1 frees V_e and K_(e+1) with one commit, so load
-      // j is freed by event (j + 1) / 2.  Event r arrives on kv_release[r % 4] as its (r / 4)-th
-      // completion; the producer has always passed event r before event r + 4 can be committed.
-      int n_load = 0;
-      for (int w = 0; w < n_outer && alive; ++w) {
-        uint32_t bits = kDense ? 0u : (tile_word(0, w) | tile_word(1, w));
-        int v_dense = 0;
-        while ((kDense ? v_dense < NB : bits != 0u) && alive) {
-          int v;
-          if (kDense) {
-            v = v_dense++;
-          } else {
-            v = 32 * w + __ffs(bits) - 1;
-            bits &= bits - 1;
-          }
-          for (int kv = 0; kv < 2; ++kv) {
-            if (n_load >= C::kSlots) {          // the slot's previous load must have been released
-              const int r = (n_load - C::kSlots + 1) >> 1;
-              if (!mbar_wait(smem_u32(&ctl->kv_release[r & 3]), (uint32_t)(r >> 2) & 1u, abort_flag, status)) {
-                alive = false;
-                break;
-              }
-            }
-            ++n_load;
-            const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
-            mbar_expect_tx(fbar, C::kSlotBytes);
-            const CUtensorMap* map = kv == 0 ? &map_k : &map_v;
-            for (int a = 0; a < C::kAtoms; ++a)
-              tma_load_3d(smem_u32(sKV + slot * C::kSlotBytes + a * C::kKVAtomBytes), map, fbar, a * 64,
-                          v * BN, bh);
-            if (++slot == C::kSlots) slot = 0;
-          }
-        }
-      }
-    }
-  } else if (warp == 9) {
-    // ================================================================== MMA issuer
-    {
-      constexpr uint32_t kIdescQK = make_idesc(BN, false);
-      constexpr uint32_t kIdescPV = make_idesc(D, true);
-      bool alive = mbar_wait(smem_u32(&ctl->q_full), 0u, abort_flag, status);
-      tc_fence_after();
-      int slot = 0;
-      uint32_t phase = 0;
-      uint32_t p_parity[2] = {0u, 0u};
-      uint32_t n_pv[2] = {0u, 0u};
-
-      // descriptor words: K-major operands (Q, K) step 32 B per k-step inside a 64-column atom and
-      // one atom (rows * 128 B) every four k-steps; the MN-major V operand steps 16 rows (2048 B)
-      constexpr uint32_t kHi = desc_hi(1024);
-      const uint32_t q_lo[2] = {desc_lo(smem_u32(sQ), 16), desc_lo(smem_u32(sQ + C::kQTileBytes), 16)};
-      const uint32_t k_lo0 = desc_lo(smem_u32(sKV), 16);
-      const uint32_t v_lo0 = desc_lo(smem_u32(sKV), C::kKVAtomBytes);
-      const uint32_t s_full_bar[2] = {smem_u32(&ctl->s_full[0]), smem_u32(&ctl->s_full[1])};
-
-      auto issue_s = [&](int k, int kslot) {
-        const uint32_t qa = q_lo[k];
-        const uint32_t ka = k_lo0 + (uint32_t)kslot * (C::kSlotBytes >> 4);
-        const uint32_t d = tmem + k * 128;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off_q = ((kk >> 2) * C::kQAtomBytes + (kk & 3) * 32) >> 4;
-          const uint32_t off_k = ((kk >> 2) * C::kKVAtomBytes + (kk & 3) * 32) >> 4;
-          tc_mma_ss(d, qa + off_q, kHi, ka + off_k, kHi, kIdescQK, kk > 0 ? 1u : 0u);
-        }
-        tc_commit(s_full_bar[k]);
-      };
-      // PV in 64-key halves: the first half starts as soon as the softmax has stored the first 32
-      // packed columns of P
-      const uint32_t p_ready_bar = smem_u32(&ctl->p_ready[0][0]);     // [k][half], 8 bytes apart
-      auto issue_pv = [&](int k, int vslot) -> bool {
-        const uint32_t va = v_lo0 + (uint32_t)vslot * (C::kSlotBytes >> 4);
-        const uint32_t d = tmem + 256 + k * 128;
-        const uint32_t pa = tmem + k * 128;
-#pragma unroll
-        for (int half = 0; half < BN / 64; ++half) {
-          if (!mbar_wait(p_ready_bar + (k * 2 + half) * 8, p_parity[k], abort_flag, status)) return false;
-          tc_fence_after();
-#pragma unroll
-          for (int kk = half * 4; kk < half * 4 + 4; ++kk)
-            tc_mma_ts(d, pa + kk * 8, va + kk * (2048 >> 4), kHi, kIdescPV, (n_pv[k] > 0 || kk > 0) ? 1u : 0u);
-        }
-        ++n_pv[k];
-        return true;
-      };
-      auto advance = [&]() {
-        if (++slot == C::kSlots) {
-          slot = 0;
-          phase ^= 1u;
-        }
-      };
-
-      // walk the union list with one entry of look-ahead
-      int w = 0;
-      uint32_t bits0 = 0, bits1 = 0;      // remaining bits of the current word, per tile
-      auto next_entry = [&](bool& h0, bool& h1) -> bool {
-        if (kDense) {                       // w counts key blocks
-          if (w >= NB) return false;
-          ++w;
-          h0 = true;
-          h1 = tile1_on;
-          return true;
-        } else {
-          while (true) {
-            const uint32_t u = bits0 | bits1;
-            if (u) {
-              const uint32_t low = u & (0u - u);
-              h0 = (bits0 & low) != 0;
-              h1 = (bits1 & low) != 0;
-              bits0 &= ~low;
-              bits1 &= ~low;
-              return true;
-            }
-            if (w >= n_words) return false;
-            bits0 = tile_word(0, w);
-            bits1 = tile_word(1, w);
-            ++w;
-          }
-        }
-      };
-
-      bool h[2], hn[2];
-      bool have = alive && next_entry(h[0], h[1]);
-      if (have) {
-        // first K tile
-        alive = mbar_wait(smem_u32(&ctl->kv_full[slot]), phase, abort_flag, status);
-        if (alive) {
-          tc_fence_after();
-          for (int k = 0; k < 2; ++k)
-            if (h[k]) issue_s(k, slot);
-          tc_commit(smem_u32(&ctl->kv_release[0]));        // release event 0: K0
-          advance();
-        }
-      }
-      uint32_t n_release = 1;
-      while (have && alive) {
-        const int vslot = slot;
-        const uint32_t vphase = phase;
-        advance();
-        const int kslot = slot;
-        const uint32_t kphase = phase;
-        const bool have_next = next_entry(hn[0], hn[1]);
-        bool v_ready = false, k_ready = false;
-        for (int k = 0; k < 2 && alive; ++k) {
-          if (h[k]) {
-            if (!v_ready) {
-              alive = mbar_wait(smem_u32(&ctl->kv_full[vslot]), vphase, abort_flag, status);
-              v_ready = true;
-            }
-            if (alive) alive = issue_pv(k, vslot);
-            if (!alive) break;
-            p_parity[k] ^= 1u;
-          }
-          if (have_next && hn[k]) {
-            if (!k_ready) {
-              alive = mbar_wait(smem_u32(&ctl->kv_full[kslot]), kphase, abort_flag, status);
-              k_ready = true;
-              if (!alive) break;
-              tc_fence_after();
-            }
-            issue_s(k, kslot);
-          }
-        }
-        if (!alive) break;
-        tc_commit(smem_u32(&ctl->kv_release[n_release & 3u]));   // V of this entry and K of the next
-        ++n_release;
-        if (have_next) advance();
-        have = have_next;
-        h[0] = hn[0];
-        h[1] = hn[1];
-      }
-      // make sure every MMA has retired before tensor memory is released
-      tc_commit(smem_u32(&ctl->drain));
-      mbar_wait(smem_u32(&ctl->drain), 0u, abort_flag, status);
-    }
-  }
-  } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
-    // ================================================================== softmax + epilogue
-    const int k = warp >> 2;                         // query tile
-    const int r = tid & (kTileM - 1);                // row inside the tile
-    const int row = q_base + k * kTileM + r;
-    const bool row_valid = row < N;
-    const int g_own = k * C::kGroups + r / BN;
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const uint32_t t_s = tmem + lane_base + k * 128;
-    const uint32_t t_o = tmem + lane_base + 256 + k * 128;
-
-    float m = -INFINITY, l = 0.f, a = 0.f;
-    float l_exact = 0.f;          // unrounded row sum (entropy kernels only)
-    // token mask: this query's coordinate and its row of the threshold table (video queries only)
-    bool tm_row = false;
-    int qx = 0, qy = 0, qt = 0;
-    const int32_t* th_row = nullptr;
-    if (kTokenMask && row < tm.n_video) {
-      const uint32_t c = tm.coord_packed[row];
-      qx = tra_coord_x(c);
-      qy = tra_coord_y(c);
-      qt = tra_coord_t(c);
-      th_row = tm.theta + (int)tm.ridx[(size_t)bh * N + row] * tm.T;
-      tm_row = true;
-    }
-    uint32_t n = 0;               // key blocks this tile has processed
-    uint32_t s_parity = 0;
-    bool alive = true;
-
-    const int n_dense = (k == 0 || tile1_on) ? NB : 0;
-    for (int w = 0; w < n_outer && alive; ++w) {
-      uint32_t bits = kDense ? 0u : tile_word(k, w);
-      const uint32_t own_bits = kDense ? 0u : ctl->bitmap[g_own][w];
-      int v_dense = 0;
-      while (kDense ? v_dense < n_dense : bits != 0u) {
-        int v;
-        bool active = true;      // a tile that is one query block retains every block of its list
-        if (kDense) {
-          v = v_dense++;
-        } else {
-          const uint32_t low = bits & (0u - bits);
-          bits &= ~low;
-          v = 32 * w + __ffs(low) - 1;
-          if (C::kGroups > 1) active = (own_bits & low) != 0;
-        }
-        const int col_limit = min(BN, N - v * BN);
-
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl->s_full[k]), s_parity, abort_flag, status))) {
-          alive = false;
-          break;
-        }
-        tc_fence_after();
-
-        // the whole S row of this thread, straight into registers (one load latency)
-        uint32_t sb[BN];
-#pragma unroll
-        for (int c = 0; c < BN / 32; ++c) tmem_ld32(t_s + c * 32, &sb[c * 32]);
-        tmem_wait_ld(&sb[0]);
-#pragma unroll
-        for (int c = 1; c < BN / 32; ++c) reg_fence32(&sb[c * 32]);
-
-        if (col_limit < BN) {          // ragged last key block: columns >= col_limit do not exist
-#pragma unroll
-          for (int j = 0; j < BN; ++j)
-            if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
-        }
-        if (kTokenMask && tm_row && active && v * BN < tm.n_video) {
-          // keys outside this query's disk at their frame distance do not exist for it (Eq. 15);
-          // text keys (index >= n_video) stay visible
-          const int k0 = v * BN;
-          const int kt0 = tra_coord_t(tm.coord_packed[k0]);
-          const int th0 = __ldg(th_row + abs(qt - kt0));
-          const int th1 = kt0 + 1 < tm.T ? __ldg(th_row + abs(qt - kt0 - 1)) : th0;
-          const uint4* kc4 = reinterpret_cast<const uint4*>(tm.coord_packed + k0);
-          const bool one_frame = k0 + BN <= tm.n_video && tra_coord_t(tm.coord_packed[k0 + BN - 1]) == kt0;
-          // 16-key slices of the block; the usual case: each is 16 consecutive x of one frame row
-          uint32_t sl[BN / 16];
-#pragma unroll
-          for (int q = 0; q < BN / 64; ++q) {
-            const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(tm.slice + (k0 >> 4)) + q);
-            sl[4 * q] = w4.x;
-            sl[4 * q + 1] = w4.y;
-            sl[4 * q + 2] = w4.z;
-            sl[4 * q + 3] = w4.w;
-          }
-          uint32_t all_runs = sl[0];
-#pragma unroll
-          for (int q = 1; q < BN / 16; ++q) all_runs &= sl[q];
-          if (all_runs & (1u << 30)) {
-            // A key (x0 + j, ys) is inside the disk iff |x0 + j - qx| <= w with
-            // w = floor(sqrt(theta - (ys - qy)^2)): one square root per slice, then an unsigned
-            // range test per key:  0 <= j + (x0 - qx + w) <= 2 w.
-#pragma unroll
-            for (int q = 0; q < BN / 16; ++q) {
-              const int ts = (int)((sl[q] >> 20) & 1023u), dts = ts - kt0;
-              const int th = dts == 0 ? th0 : (dts == 1 ? th1 : __ldg(th_row + abs(qt - ts)));
-              const int dy = tra_coord_y(sl[q]) - qy;
-              const int rem = th - dy * dy;
-              const int w = tra_isqrt_small_nocvt(max(rem, 0));
-              const uint32_t base = rem < 0 ? 0x40000000u : (uint32_t)(w + tra_coord_x(sl[q]) - qx);
-              const uint32_t span = (uint32_t)(2 * w);
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (base + (uint32_t)j > span) sb[q * 16 + j] = __float_as_uint(-1e30f);
-            }
-          } else if (one_frame) {       // every key of the block in one frame, some slice not a row run
-#pragma unroll
-            for (int j4 = 0; j4 < BN / 4; ++j4) {
-              const uint4 c4 = __ldg(kc4 + j4);
-              const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
-#pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4) {
-                const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
-                if (dx * dx + dy * dy > th0) sb[j4 * 4 + q4] = __float_as_uint(-1e30f);
-              }
-            }
-          } else {
-#pragma unroll
-            for (int j4 = 0; j4 < BN / 4; ++j4) {
-              const uint4 c4 = __ldg(kc4 + j4);
-              const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
-#pragma unroll
-              for (int q4 = 0; q4 < 4; ++q4) {
-                const int j = j4 * 4 + q4;
-                const int dt = tra_coord_t(cs[q4]) - kt0;
-                const int th = dt == 0 ? th0 : (dt == 1 ? th1 : __ldg(th_row + abs(qt - kt0 - dt)));
-                const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
-                if (k0 + j < tm.n_video && dx * dx + dy * dy > th) sb[j] = __float_as_uint(-1e30f);
-              }
-            }
-          }
-        }
-        float alpha = 1.f;
-        bool row_on = active;         // false also when the token mask leaves this row nothing here
-        if (active) {
-          float mx0 = __uint_as_float(sb[0]), mx1 = __uint_as_float(sb[1]);
-#pragma unroll
-          for (int j = 2; j + 3 < BN; j += 4) {
-            mx0 = fmax3(mx0, __uint_as_float(sb[j]), __uint_as_float(sb[j + 1]));
-            mx1 = fmax3(mx1, __uint_as_float(sb[j + 2]), __uint_as_float(sb[j + 3]));
-          }
-          mx0 = fmax3(mx0, __uint_as_float(sb[BN - 2]), __uint_as_float(sb[BN - 1]));
-          const float mx = fmaxf(mx0, mx1);
-          if (kTokenMask) row_on = mx > -1e29f;
-          const float m_blk = mx * scale_log2;
-          if (row_on && m_blk > m + kRescaleThreshold) {   // also the first block (m = -inf)
-            alpha = ex2(m - m_blk);                   // 0 when m = -inf
-            a = l_exact > 0.f ? alpha * (a + (m - m_blk) * l_exact) : 0.f;
-            l *= alpha;
-            l_exact *= alpha;
-            m = m_blk;
-          }
-        }
-        // rescale the O accumulator when some row of this warp raised its reference maximum
-        const bool warp_rescale = __any_sync(0xffffffffu, alpha != 1.f) && n > 0;
-        if (warp_rescale) {
-          // PV(n-1) of this tile has retired: the S the thread just read was issued behind it on
-          // the same in-order pipe, and the commit that announced S covers every earlier MMA
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t o[32];
-            tmem_ld32(t_o + c * 32, o);
-            tmem_wait_ld(o);
-#pragma unroll
-            for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
-            tmem_st32(t_o + c * 32, o);
-          }
-        }
-        // probabilities (relative to m), row sum and entropy accumulator; P goes back to tensor
-        // memory 32 keys at a time, and each 64-key half is announced to the MMA issuer on its own
-        {
-          const float neg_m = row_on ? -m : 0.f;
-          const uint64_t scale2 = pack2(scale_log2, scale_log2), neg_m2 = pack2(neg_m, neg_m);
-          uint64_t l2 = 0ull, a2 = 0ull, e2 = 0ull;      // pairs of partial sums
-#pragma unroll
-          for (int c = 0; c < BN / 32; ++c) {
-            uint32_t pk[16];
-            if (active) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 2) {
-                const uint64_t t2 = ffma2(pack2(__uint_as_float(sb[c * 32 + j]), __uint_as_float(sb[c * 32 + j + 1])),
-                                          scale2, neg_m2);
-                float t0, t1, x0, x1;
-                unpack2(t2, t0, t1);
-                x0 = ex2(t0);
-                x1 = ex2(t1);
-                // the row sum that normalises O uses the bf16-rounded probabilities the PV MMA
-                // consumes, so numerator and denominator of O = (sum p v) / (sum p) agree
-                const uint32_t packed = pack_bf16(x0, x1);
-                l2 = fadd2(l2, pack2(__uint_as_float(packed << 16), __uint_as_float(packed & 0xffff0000u)));
-                if (kEntropy) {               // entropy and lse from the unrounded terms
-                  const uint64_t x2 = pack2(x0, x1);
-                  e2 = fadd2(e2, x2);
-                  a2 = ffma2(x2, t2, a2);
-                }
-                pk[j >> 1] = packed;
-              }
-            } else {                          // this row's query block does not retain the key block
-#pragma unroll
-              for (int j = 0; j < 16; ++j) pk[j] = 0u;
-            }
-            tmem_st16(t_s + c * 16, pk);
-            if (c & 1) {                      // a 64-key half of P is complete
-              tmem_wait_st();
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(smem_u32(&ctl->p_ready[k][c >> 1]));
-            }
-          }
-          float lo, hi;
-          unpack2(l2, lo, hi);
-          l += lo + hi;
-          if (kEntropy) {
-            unpack2(a2, lo, hi);
-            a += lo + hi;
-            unpack2(e2, lo, hi);
-            l_exact += lo + hi;
-          }
-        }
-        s_parity ^= 1u;
-        ++n;
-      }
-    }
-
-    // ---- epilogue: O = o / l, entropy, lse ------------------------------------------------
-    // the MMA warp commits `drain` behind its last MMA: every PV of both tiles has retired then
-    if (alive && n > 0)
-      alive = __all_sync(0xffffffffu, mbar_wait(smem_u32(&ctl->drain), 0u, abort_flag, status));
-    if (alive) {
-      tc_fence_after();
-      const float inv_l = l > 0.f ? 1.f / l : 0.f;
-      __nv_bfloat16* orow = O + ((size_t)bh * N + (row_valid ? row : 0)) * D;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t o_bits[32];
-        float o[32];
-        if (n > 0) {
-          tmem_ld32(t_o + c * 32, o_bits);
-          tmem_wait_ld(o_bits);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] = __uint_as_float(o_bits[j]);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) o[j] = 0.f;
-        }
-        if (row_valid) {
-          uint4* dst = (uint4*)(orow + c * 32);
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) {
-            uint4 val;
-            val.x = pack_bf16(o[q4 * 8 + 0] * inv_l, o[q4 * 8 + 1] * inv_l);
-            val.y = pack_bf16(o[q4 * 8 + 2] * inv_l, o[q4 * 8 + 3] * inv_l);
-            val.z = pack_bf16(o[q4 * 8 + 4] * inv_l, o[q4 * 8 + 5] * inv_l);
-            val.w = pack_bf16(o[q4 * 8 + 6] * inv_l, o[q4 * 8 + 7] * inv_l);
-            dst[q4] = val;
-          }
-        }
-      }
-      if (row_valid) {
-        const size_t idx = (size_t)bh * N + row;
-        const float l_out = kEntropy ? l_exact : l;
-        if (kEntropy && entropy) entropy[idx] = l_out > 0.f ? logf(l_out) - kLn2 * a / l_out : 0.f;
-        if (lse) lse[idx] = l_out > 0.f ? (m + log2f(l_out)) * kLn2 : -INFINITY;
-      }
-    }
-  }
-
-  // ---- teardown ------------------------------------------------------------------------
-  tc_fence_before();
-  __syncthreads();
-  if (warp == 9) {
-    if (ctl->abort_flag) {
-      // let copies and MMAs that were in flight when the CTA gave up land before releasing
-      const unsigned long long t0 = globaltimer_ns();
-      while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-    }
-    tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem) : "memory");
-  }
-}
-
-// ------------------------------------------------------------------------------------ host
-typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                    const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-encode_tiled_fn get_encode_tiled() {
-  static encode_tiled_fn fn = nullptr;
-  if (!fn) {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = (encode_tiled_fn)p;
-  }
-  return fn;
-}
-
-// [B*heads, N, d] bf16 viewed as a 3-D tensor (d innermost); box = 64 columns x `rows` tokens.
-int make_map(CUtensorMap* map, const void* base, int d, int N, long long BH, int rows) {
-  encode_tiled_fn enc = get_encode_tiled();
-  if (!enc) return TRA_ERR_CUDA;
-  cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)N, (cuuint64_t)BH};
-  cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)d * 2 * (cuuint64_t)N};
-  cuuint32_t box[3] = {64u, (cuuint32_t)rows, 1u};
-  cuuint32_t estr[3] = {1u, 1u, 1u};
-  CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
-                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? TRA_OK : TRA_ERR_CUDA;
-}
-
-template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense>
-int launch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O, float* entropy,
-           float* lse, const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, long long BH,
-           float sm_scale, cudaStream_t stream) {
-  using C = Cfg<D, BN>;
-  CUtensorMap mq, mk, mv;
-  int rc;
-  if ((rc = make_map(&mq, Q, D, plan->S, BH, kTileM)) != TRA_OK) return rc;
-  if ((rc = make_map(&mk, K, D, plan->S, BH, BN)) != TRA_OK) return rc;
-  if ((rc = make_map(&mv, V, D, plan->S, BH, BN)) != TRA_OK) return rc;
-  auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense>;
-  TokenMaskArgs tm = {plan->d_boxes, plan->d_slice, plan->d_coord_packed, plan->d_theta, ridx, plan->N, plan->cfg.T};
-  TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-  const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
-  dim3 grid((unsigned)n_pairs, (unsigned)BH);
-  kern<<<grid, kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, (__nv_bfloat16*)O, entropy, lse, row_ptr,
-                                                  col_idx, plan->S, plan->NB, sm_scale * kLog2e,
-                                                  plan->d_status, tm);
-  TRA_CUDA_CHECK(cudaGetLastError());
-  return TRA_OK;
-}
-
 int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const void* V, void* O,
                   float* entropy, float* lse, const int32_t* row_ptr, const int32_t* col_idx,
-                  const uint16_t* ridx, int B, int heads, float sm_scale, void* stream_) {
+                  const uint16_t* ridx, const int32_t* tile_pairs, int B, int heads, float sm_scale,
+                  void* stream_) {
   if (!plan || !Q || !K || !V || !O || B < 1 || heads < 1) return TRA_ERR_INVALID_ARG;
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)V | (uintptr_t)O) & 127) return TRA_ERR_INVALID_ARG;
   if (!(sm_scale > 0.f)) return TRA_ERR_INVALID_ARG;
   const long long BH = (long long)B * heads;
   if (BH > 65535 || plan->NB > 32 * kMaxBitmapWords) return TRA_ERR_UNSUPPORTED;
-  cudaStream_t stream = (cudaStream_t)stream_;
+  if (entropy != nullptr && (row_ptr != nullptr || ridx != nullptr)) return TRA_ERR_INVALID_ARG;
+  const tra_attn_args a = {plan, Q,   K,          V,  O,        entropy,
+                           lse,  row_ptr, col_idx, ridx, tile_pairs, BH, sm_scale, (cudaStream_t)stream_};
   const int d = plan->cfg.head_dim, b = plan->cfg.block;
-  // entropy launches are dense, token-mask launches block-sparse; a plain launch may be either
-  const int variant = (entropy != nullptr ? 1 : 0) + (ridx != nullptr ? 2 : 0);   // never 3
-  if (variant == 1 && row_ptr != nullptr) return TRA_ERR_INVALID_ARG;
-#define TRA_ATTN_CASE(DD, BB)                                                                          \
-  if (d == DD && b == BB) {                                                                            \
-    if (variant == 1)                                                                                  \
-      return launch<DD, BB, true, false, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, \
-                                               BH, sm_scale, stream);                                  \
-    if (variant == 2)                                                                                  \
-      return launch<DD, BB, false, true, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx,      \
-                                                ridx, BH, sm_scale, stream);                           \
-    if (row_ptr == nullptr)                                                                            \
-      return launch<DD, BB, false, false, true>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx,      \
-                                                ridx, BH, sm_scale, stream);                           \
-    return launch<DD, BB, false, false, false>(plan, Q, K, V, O, entropy, lse, row_ptr, col_idx, ridx, \
-                                               BH, sm_scale, stream);                                  \
-  }
-  TRA_ATTN_CASE(128, 128)
-  TRA_ATTN_CASE(64, 64)
-  TRA_ATTN_CASE(64, 128)
-  TRA_ATTN_CASE(128, 64)
-#undef TRA_ATTN_CASE
+  if (d == 128 && b == 128) return tra_attn_launch_d128_b128(a);
+  if (d == 64 && b == 64) return tra_attn_launch_d64_b64(a);
+  if (d == 64 && b == 128) return tra_attn_launch_d64_b128(a);
+  if (d == 128 && b == 64) return tra_attn_launch_d128_b64(a);
   return TRA_ERR_UNSUPPORTED;
 }
 
@@ -1016,13 +50,16 @@ extern "C" int tra_selftest_wait_timeout(tra_plan_t* plan, int limit_ms, void* s
 extern "C" int tra_entropy_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
                                 void* O, float* entropy, float* lse, int B, int heads, float sm_scale,
                                 void* stream) {
-  return attn_dispatch(plan, Q, K, V, O, entropy, lse, nullptr, nullptr, nullptr, B, heads, sm_scale, stream);
+  return attn_dispatch(plan, Q, K, V, O, entropy, lse, nullptr, nullptr, nullptr, nullptr, B, heads, sm_scale,
+                       stream);
 }
 
 extern "C" int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const void* V,
-                               const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx, void* O,
-                               float* lse, int B, int heads, float sm_scale, void* stream) {
+                               const int32_t* row_ptr, const int32_t* col_idx, const uint16_t* ridx,
+                               const int32_t* tile_pairs, void* O, float* lse, int B, int heads, float sm_scale,
+                               void* stream) {
   // a block list, or (with ridx) none at all: Eq. 16 itself
   if ((row_ptr == nullptr) != (col_idx == nullptr) || (!row_ptr && !ridx)) return TRA_ERR_INVALID_ARG;
-  return attn_dispatch(plan, Q, K, V, O, nullptr, lse, row_ptr, col_idx, ridx, B, heads, sm_scale, stream);
+  return attn_dispatch(plan, Q, K, V, O, nullptr, lse, row_ptr, col_idx, ridx, tile_pairs, B, heads, sm_scale,
+                       stream);
 }

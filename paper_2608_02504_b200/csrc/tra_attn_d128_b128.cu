@@ -1,0 +1,4 @@
+// Attention kernels for head_dim 128, block 128.
+#include "tra_attn_kernel.cuh"
+
+int tra_attn_launch_d128_b128(const tra_attn_args& a) { return launch_shape<128, 128>(a); }

@@ -1,0 +1,4 @@
+// Attention kernels for head_dim 64, block 128.
+#include "tra_attn_kernel.cuh"
+
+int tra_attn_launch_d64_b128(const tra_attn_args& a) { return launch_shape<64, 128>(a); }

@@ -15,7 +15,7 @@ size_t align_up(size_t x) { return (x + kAlign - 1) & ~(kAlign - 1); }
 
 // Device buffers of one pass, carved from the caller's workspace.
 struct HostPassLayout {
-  size_t stage_in[2][3], stage_out[2], qkv[3], o_dense, o_sparse, entropy, ridx, mask, row_ptr, col_idx, nnz;
+  size_t stage_in[2][3], stage_out[2], qkv[3], o_dense, o_sparse, entropy, ridx, mask, row_ptr, col_idx, nnz, pairs;
   size_t total;
 };
 
@@ -41,6 +41,7 @@ HostPassLayout make_layout(const tra_plan_t* plan, int group) {
   L.row_ptr = take((g * NB + 1) * 4);
   L.col_idx = take(g * NB * NB * 4);
   L.nnz = take(8);
+  L.pairs = take(g * (((S + 127) / 128 + 1) / 2) * 2 * 4);
   L.total = off;
   return L;
 }
@@ -136,10 +137,11 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
       return rc;
     if ((rc = tra_build_block_mask(plan, (const uint16_t*)(ws + L.ridx), ws + L.mask, (int32_t*)(ws + L.row_ptr),
                                    (int32_t*)(ws + L.col_idx), (int64_t)((size_t)n * NB * NB),
-                                   (int64_t*)(ws + L.nnz), 1, n, cs)) != TRA_OK)
+                                   (int64_t*)(ws + L.nnz), (int32_t*)(ws + L.pairs), 1, n, cs)) != TRA_OK)
       return rc;
     if ((rc = tra_sparse_attn(plan, Q, K, V, (const int32_t*)(ws + L.row_ptr), (const int32_t*)(ws + L.col_idx),
-                              nullptr, ws + L.o_sparse, nullptr, 1, n, sm_scale, cs)) != TRA_OK)
+                              nullptr, (const int32_t*)(ws + L.pairs), ws + L.o_sparse, nullptr, 1, n, sm_scale,
+                              cs)) != TRA_OK)
       return rc;
     if (out_free[b]) TRA_CUDA_CHECK(cudaStreamWaitEvent(cs, out_free[b], 0));
     if ((rc = tra_tile_major_scatter(plan, ws + L.o_sparse, ws + L.stage_out[b], n, row_bytes, cs)) != TRA_OK)

@@ -44,7 +44,7 @@ __global__ void __launch_bounds__(TRA_MASK_THREADS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
                       uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int S, int NB,
-                      int NBv, int b, int T, int H, int W, int keep_diagonal) {
+                      int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal) {
   extern __shared__ int32_t s_dyn[];
   __shared__ int s_rank_ridx[128];
   __shared__ tra_block_boxes_t s_ubox;
@@ -64,7 +64,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   const uint16_t* ridx_h = ridx + bh * S;
   uint8_t* mask_row = block_mask + (bh * NB + u) * (long long)NB;
 
-  // Text rows (u >= NBv) keep every block (Algorithm 1: "text or non-video blocks remain dense").
+  // Rows of text blocks (u >= NBv) keep every block: Algorithm 1 leaves non-video blocks dense.
   if (u >= NBv) {
     for (int v = tid; v < NB; v += TRA_MASK_THREADS) mask_row[v] = 1;
     if (tid == 0) row_ptr[bh * NB + u + 1] = NB;
@@ -82,7 +82,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     qx = tra_coord_x(c);
     qy = tra_coord_y(c);
     qt = tra_coord_t(c);
-    qr = ridx_h[q0 + tid];
+    qr = min((int)ridx_h[q0 + tid], n_radii - 1);      // a candidate index past the table reads its last row
     s_rank_ridx[tid] = qr;
   }
   if (tid == 0) {
@@ -264,7 +264,10 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
 }
 
 // ---------------------------------------------------------------------------------------
-// In-place exclusive scan of the per-row counts held in row_ptr[1..rows] (one CTA).
+// In-place exclusive scan of the per-row counts held in row_ptr[1..rows] (one CTA).  When the
+// total exceeds the capacity of col_idx every offset is clamped to the capacity, so that a
+// later attention launch that reads col_idx[row_ptr[r] .. row_ptr[r+1]) stays inside the buffer
+// (rows past the capacity come out short or empty; the error is in the plan status).
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 tra_row_ptr_scan_kernel(int32_t* __restrict__ row_ptr, long long rows, long long capacity,
@@ -285,9 +288,10 @@ tra_row_ptr_scan_kernel(int32_t* __restrict__ row_ptr, long long rows, long long
   }
   long long run = s_part[tid] - sum;                   // exclusive prefix of this chunk
   const long long total = s_part[1023];
+  const long long cap = min(capacity, 0x7fffffffll);
   for (long long i = lo; i < hi; ++i) {
     run += row_ptr[i + 1];
-    row_ptr[i + 1] = (int32_t)run;
+    row_ptr[i + 1] = (int32_t)min(run, cap);
   }
   if (tid == 0) {
     row_ptr[0] = 0;
@@ -319,9 +323,113 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Tile pairing for the block-sparse attention launch.  That launch gives every CTA two 128-row
+// query tiles which walk the union of their key-block lists; a key block only one of the two
+// retains leaves the other tile idle.  This kernel pairs tiles with similar lists: one CTA per
+// (batch, head); tile t covers the query blocks [t G, (t + 1) G), G = 128 / block.
+//   1. row bitmaps of a window of tiles are built in shared memory (ballots over the byte mask),
+//      and for every tile u the number of key blocks that u and u + 1 + c do not share is
+//      stored for c = 0 .. kPairWindow - 1;
+//   2. one warp matches the tiles greedily in ascending order: the first unmatched tile takes the
+//      unmatched tile of its window with the fewest unshared key blocks, or, when the window has
+//      none left, the next unmatched tile after it.  Every tile is matched (one is left alone
+//      when their number is odd): pairs[i] = (u, v) for i < ceil(NT / 2), v = -1 for a lone tile.
+// Any perfect matching gives the same attention output; the choice only moves time.
+// ---------------------------------------------------------------------------------------
+#define TRA_PAIR_WINDOW 8
+#define TRA_PAIR_CHUNK 32
+#define TRA_PAIR_THREADS 256
+
+__global__ void __launch_bounds__(TRA_PAIR_THREADS)
+tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restrict__ pairs, int NB, int NT, int G) {
+  extern __shared__ uint32_t s_pair[];
+  const int words = (NB + 31) >> 5;
+  const int win_rows = TRA_PAIR_CHUNK + TRA_PAIR_WINDOW;
+  uint32_t* s_win = s_pair;                                                  // [win_rows][words]
+  uint16_t* s_band = (uint16_t*)(s_win + win_rows * words);                  // [NT][window]
+  uint8_t* s_used = (uint8_t*)(s_band + (size_t)NT * TRA_PAIR_WINDOW);       // [NT]
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long bh = blockIdx.x;
+  const uint8_t* mask_h = block_mask + bh * NB * (long long)NB;
+  int32_t* out = pairs + bh * ((NT + 1) / 2) * 2;
+
+  for (int t = tid; t < NT; t += TRA_PAIR_THREADS) s_used[t] = 0;
+  for (int chunk0 = 0; chunk0 < NT; chunk0 += TRA_PAIR_CHUNK) {
+    const int rows = min(win_rows, NT - chunk0);
+    __syncthreads();                         // the previous chunk's window has been read
+    // one warp per window row; the loads of eight words of the row are in flight together
+    for (int r = warp; r < rows; r += TRA_PAIR_THREADS / 32) {
+      for (int wd0 = 0; wd0 < words; wd0 += 8) {
+        uint32_t on[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+        for (int g = 0; g < G; ++g) {
+          const int u = (chunk0 + r) * G + g;
+          if (u >= NB) break;
+          const uint8_t* row = mask_h + (long long)u * NB;
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {           // eight independent loads
+            const int j = (wd0 + q) * 32 + lane;
+            on[q] |= j < NB ? (uint32_t)row[j] : 0u;
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const uint32_t bits = __ballot_sync(0xffffffffu, on[q] != 0u);
+          if (lane == 0 && wd0 + q < words) s_win[r * words + wd0 + q] = bits;
+        }
+      }
+    }
+    __syncthreads();
+    for (int task = tid; task < TRA_PAIR_CHUNK * TRA_PAIR_WINDOW; task += TRA_PAIR_THREADS) {
+      const int ul = task / TRA_PAIR_WINDOW, c = task - ul * TRA_PAIR_WINDOW;
+      const int u = chunk0 + ul, v = u + 1 + c;
+      if (u >= NT) continue;
+      uint32_t d = 0xffffu;
+      if (v < NT) {
+        d = 0;
+        const uint32_t* a = s_win + ul * words;
+        const uint32_t* b = s_win + (ul + 1 + c) * words;
+        for (int wd = 0; wd < words; ++wd) d += __popc(a[wd] ^ b[wd]);
+        d = min(d, 0xfffeu);
+      }
+      s_band[u * TRA_PAIR_WINDOW + c] = (uint16_t)d;
+    }
+  }
+  __syncthreads();
+  if (warp != 0) return;
+  int n_out = 0;
+  for (int u = 0; u < NT; ++u) {
+    if (s_used[u]) continue;                 // the same for every lane
+    uint32_t key = 0xffffffffu;              // (unshared blocks, window position) of this lane's candidate
+    if (lane < TRA_PAIR_WINDOW) {
+      const int v = u + 1 + lane;
+      if (v < NT && !s_used[v]) key = ((uint32_t)s_band[u * TRA_PAIR_WINDOW + lane] << 8) | (uint32_t)lane;
+    }
+    key = __reduce_min_sync(0xffffffffu, key);
+    int v = -1;
+    if (key != 0xffffffffu) {
+      v = u + 1 + (int)(key & 0xffu);
+    } else {                                 // nothing left in the window: the next unmatched tile, if any
+      for (int base = u + 1 + TRA_PAIR_WINDOW; base < NT && v < 0; base += 32) {
+        const int cand = base + lane;
+        const uint32_t free_mask = __ballot_sync(0xffffffffu, cand < NT && !s_used[cand]);
+        if (free_mask) v = base + __ffs(free_mask) - 1;
+      }
+    }
+    if (lane == 0) {
+      s_used[u] = 1;
+      if (v >= 0) s_used[v] = 1;
+      out[2 * n_out] = u;
+      out[2 * n_out + 1] = v;
+    }
+    ++n_out;
+    __syncwarp();
+  }
+}
+
 extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* block_mask,
                                     int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
-                                    int64_t* nnz_out, int B, int heads, void* stream_) {
+                                    int64_t* nnz_out, int32_t* tile_pairs, int B, int heads, void* stream_) {
   if (!plan || !ridx || !block_mask || !row_ptr || !col_idx || B < 1 || heads < 1 ||
       col_idx_capacity < 0)
     return TRA_ERR_INVALID_ARG;
@@ -341,8 +449,7 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
                                         (int)smem));
   tra_block_vote_kernel<<<grid, TRA_MASK_THREADS, smem, stream>>>(
       ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, plan->S, NB,
-      plan->NBv,
-      plan->cfg.block, T, H, W, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
+      plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,
                                                   plan->d_status);
@@ -350,5 +457,20 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   tra_col_idx_fill_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(
       block_mask, row_ptr, col_idx, rows, NB, (long long)col_idx_capacity);
   TRA_CUDA_CHECK(cudaGetLastError());
+  if (tile_pairs) {
+    // query tiles of the attention launch: 128 rows = G blocks (block sizes that do not divide 128
+    // have no attention kernel; their table pairs consecutive "tiles" of one block each)
+    const int b = plan->cfg.block;
+    const int G = (128 % b == 0) ? 128 / b : 1;
+    const int NT = (NB + G - 1) / G;
+    const size_t pair_smem = ((size_t)(TRA_PAIR_CHUNK + TRA_PAIR_WINDOW) * ((NB + 31) / 32)) * 4 +
+                             (size_t)NT * TRA_PAIR_WINDOW * 2 + (size_t)NT;
+    if (pair_smem > 200 * 1024) return TRA_ERR_UNSUPPORTED;
+    if (pair_smem > 48 * 1024)
+      TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)pair_smem));
+    tra_pair_tiles_kernel<<<(unsigned)BH, TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G);
+    TRA_CUDA_CHECK(cudaGetLastError());
+  }
   return TRA_OK;
 }

@@ -8,7 +8,7 @@
 #include "tra_common.cuh"
 
 // ---------------------------------------------------------------------------------------
-// Count table C_grid (Eq. 13; "stored in a lookup table", Section 3.2).
+// Count table C_grid (Eq. 13), the per-coordinate lookup table of Section 3.2.
 // One thread per (y, x, candidate k).  The in-frame count
 //   A(theta) = #{(y', x') : (y'-y)^2 + (x'-x)^2 <= theta}
 // is a sweep over rows: each row contributes the clipped length of an x-interval.

@@ -38,7 +38,8 @@ def test_status_strings_and_null_arguments():
     assert lib.tra_plan_create(None, None, None) == -1
     assert lib.tra_plan_destroy(None) == -1
     assert lib.tra_budget_radius(None, None, None, None, None, 1, 1, None) == -1
-    assert lib.tra_sparse_attn(None, None, None, None, None, None, None, None, None, 1, 1, ctypes.c_float(1.0), None) == -1
+    assert lib.tra_sparse_attn(None, None, None, None, None, None, None, None, None, None, 1, 1, ctypes.c_float(1.0),
+                               None) == -1
     assert lib.tra_entropy_attn(None, None, None, None, None, None, None, 1, 1, ctypes.c_float(1.0), None) == -1
     lib.tra_hot_path_host_workspace_bytes.restype = ctypes.c_size_t
     assert lib.tra_hot_path_host_workspace_bytes(None, 8) == 0

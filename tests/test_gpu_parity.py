@@ -238,10 +238,28 @@ def test_block_mask_capacity_error_is_reported():
     plan = make_plan(cfg)
     full = np.full((1, geo.N), geo.radii.size - 1, np.uint16)
     ridx = torch.from_numpy(full.view(np.int16)).to(DEV)[None]
-    small = torch.empty(3, dtype=torch.int32, device=DEV)
-    plan.build_block_mask(ridx, col_idx=small)
+    small = torch.full((3 + 64,), -7, dtype=torch.int32, device=DEV)      # 3 entries of capacity, then a guard zone
+    _, row_ptr, _, nnz = plan.build_block_mask(ridx, col_idx=small[:3])
+    # an asynchronous caller chains the attention call before it reads the status: the list offsets
+    # are clamped to the capacity, so the kernel stays inside col_idx
+    Q, K, V = tile_major_inputs(cfg, plan, heads=[0])
+    O, _ = plan.sparse_attn(Q, K, V, row_ptr, small[:3])
     assert plan.status() == -3          # TRA_ERR_CAPACITY
     assert plan.status() == 0           # cleared by the read
+    rp = row_ptr.cpu().numpy()
+    assert rp[0] == 0 and np.all(np.diff(rp) >= 0) and rp.max() == 3
+    assert int(nnz.item()) == geo.NB * geo.NB            # the true count is still reported
+    assert torch.all(small[3:] == -7)                   # nothing was written past the capacity
+    assert torch.isfinite(O.float()).all()
+    # candidate indices past the table are read as its last entry (full support), not out of bounds
+    wild = torch.full((1, 1, geo.N), -1, dtype=torch.int16, device=DEV)     # 65535 as uint16
+    m_wild, rp_w, ci_w, _ = plan.build_block_mask(wild)
+    m_full, _, _, _ = plan.build_block_mask(ridx)
+    assert torch.equal(m_wild, m_full)
+    Ow, _ = plan.sparse_attn(Q, K, V, rp_w, ci_w, ridx=wild)
+    Of, _ = plan.sparse_attn(Q, K, V, rp_w, ci_w, ridx=ridx)
+    plan.check_status()
+    assert torch.equal(Ow, Of)
     plan.close()
 
 
@@ -342,8 +360,8 @@ def test_sparse_attn_all_rows(cfg, kind):
         assert np.all(got[empty] == 0)                               # empty block row -> zeros
         got_lse = lse[0, h].cpu().numpy().astype(np.float64)
         assert np.all(np.isneginf(got_lse[empty]))
-        if (~empty).any():       # the sparse call forms lse from bf16-rounded probabilities
-            assert np.abs(got_lse[~empty] - ref["lse"][~empty]).max() <= 4e-3
+        if (~empty).any():
+            assert np.abs(got_lse[~empty] - ref["lse"][~empty]).max() <= 1e-3
     if kind == "small":
         assert n_empty > 0                                           # the degenerate case is exercised
     plan.close()
@@ -417,7 +435,7 @@ def test_sparse_attn_token_level_without_block_list(cfg, n_text, kind):
         assert vis2.any(axis=1).all()              # a query always sees itself
         ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis2)
         common.assert_output(O[0, h], ref["O"], f"token-level head {h}")
-        assert np.abs(lse[0, h].cpu().numpy().astype(np.float64) - ref["lse"]).max() <= 4e-3
+        assert np.abs(lse[0, h].cpu().numpy().astype(np.float64) - ref["lse"]).max() <= 1e-3
     with pytest.raises(api().TraError):
         plan.sparse_attn(Q, K, V, None, None)       # neither a block list nor radii
     plan.close()
@@ -488,7 +506,7 @@ def sampled_rows(geo, rng, n_random):
                          [("wan1.3b-480p", (0, 3, 7, 11), 100), ("wan14b-720p", (0, 13, 26, 39), 100),
                           ("hunyuan-720p", (0, 7, 15, 23), 60)])
 def test_full_size_sampled_rows(name, heads_checked, n_random):
-    """At the BASELINE shapes, all heads resident, in the launch configuration the benchmark times:
+    """At the three full-size shapes, all heads resident, in the launch configuration the benchmark times:
     sampled (head, row) pairs of dense attention + entropy, the integer stages of their block
     rows, sparse attention, and sparse attention with the token mask inside the blocks.  Rows cover the first / last blocks and the ragged tail."""
     cfg = workloads.CONFIGS[name]
@@ -702,7 +720,7 @@ def test_host_pipeline_matches_device_path():
             assert torch.equal(out, expect)
         sizes = api().HostPipeline.group_sizes(cfg["heads"], pipe.group, pipe.first_group)
         assert sum(sizes) == cfg["heads"] and max(sizes) <= pipe.group and sizes[0] <= pipe.first_group
-        assert launches == 10 * len(sizes)
+        assert launches == 11 * len(sizes)
     with pytest.raises(ValueError):
         pipe.run(Qr, host[1], host[2], out)     # a device tensor where a pinned host tensor belongs
     # the C entry point refuses a workspace that is too small or misaligned, before any work

@@ -17,18 +17,20 @@ def _worker(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
                       LOCAL_RANK=str(rank))
     import bench
-    r, w, local = bench.dist_setup(world)
+    r, w, local = bench.dist_setup()
     assert (r, w, local) == (rank, world, rank)
     bench.barrier(w)
-    # every rank times its own replica; the reported time is the slowest rank's
+    # every rank times its own share; the reported time is the slowest rank's, the work is the sum
     mine = 10.0 + 5.0 * rank
-    slowest = bench.max_over_ranks(mine, w, torch.device("cpu"))
+    slowest = bench.reduce_over_ranks(mine, w, torch.device("cpu"))
+    total = bench.reduce_over_ranks(mine, w, torch.device("cpu"), "sum")
+    assert total == 25.0
     # the path shards by head with no exchange: each rank's oracle result for its own heads equals
     # the single-process result for those heads
     import oracle
     from paper_2608_02504_b200 import workloads
     cfg = workloads.CONFIGS["tiny"]
-    heads = [h for h in range(cfg["heads"]) if h % w == r]
+    heads = list(range(cfg["heads"]))[r::w]        # what `bench.py --shard heads` gives rank r
     Q, K, V = workloads.make_qkv(cfg, "cpu", heads=heads)
     Qf, Kf, Vf = workloads.make_qkv(cfg, "cpu")
     same = all(torch.equal(a[0, i], b[0, h]) for a, b in ((Q, Qf), (K, Kf), (V, Vf)) for i, h in enumerate(heads))
@@ -57,6 +59,6 @@ def test_reference_arm_non_zero_ranks_do_nothing(monkeypatch, capsys):
     monkeypatch.setenv("RANK", "1")
 
     class A:
-        config, tau, cpu_rows, warmup, steps, gpus = "tiny", None, 128, 0, 1, 2
+        config, tau, heads, cpu_rows, warmup, steps, gpus, shard = "tiny", None, None, 128, 0, 1, 2, "replicas"
     bench.run_reference(A)
     assert capsys.readouterr().out == ""

@@ -209,6 +209,35 @@ def test_grid_count_float_sqrt_form_and_table():
                     assert counts[f, y, x, k] == oracle.grid_count_brute(T, H, W, th[k], f, y, x)
 
 
+@pytest.mark.parametrize("T,H,W", [(21, 45, 80), (33, 45, 80)])
+@pytest.mark.parametrize("gamma", [0.6, 0.95, 0.0513])
+def test_grid_count_float_sqrt_form_on_the_full_size_grids(T, H, W, gamma):
+    # Eq. 13 in its literal floating form (Euclidean distance against r exp(-gamma delta)), evaluated
+    # by numpy over every key of the real latent grids, for a centre and a corner query, against the
+    # oracle's integer-threshold enumeration.  Candidates whose decayed radius comes within 1e-9 of a
+    # lattice distance are skipped (the two forms may round a tie differently); few are.  A key at the
+    # query's own (y, x) is inside for every radius >= 0 in both forms.
+    radii = oracle.default_radii(T, H, W, gamma)
+    th = oracle.theta_table(radii, T, H, W, gamma)
+    tt, yy, xx = np.meshgrid(np.arange(T), np.arange(H), np.arange(W), indexing="ij")
+    diag = math.hypot(H - 1, W - 1)
+    checked = 0
+    for f, y, x in ((T // 2, H // 2, W // 2), (0, 0, 0), (T - 1, H - 1, 0)):
+        ds = np.sqrt((yy - y) ** 2 + (xx - x) ** 2)
+        dt = np.abs(tt - f)
+        for k in list(range(0, radii.size, 7)) + [radii.size - 1]:
+            rho = np.minimum(radii[k] * np.exp(-gamma * dt), diag)      # the frame diagonal is full support
+            near_tie = (np.abs(ds - rho) < 1e-9) & ~((dt == 0) & (ds <= rho)) & (rho < diag) & (ds > 0)
+            if near_tie.any():
+                continue
+            assert oracle.grid_count_brute(T, H, W, th[k], f, y, x) == int((ds <= rho).sum()), (f, y, x, k)
+            checked += 1
+    assert checked >= 30
+    # r = 0 keeps the query's own cell in every frame; the last candidate is full support
+    assert oracle.grid_count_brute(T, H, W, th[0], T // 2, H // 2, W // 2) == T
+    assert oracle.grid_count_brute(T, H, W, th[-1], 0, 0, 0) == T * H * W
+
+
 def test_grid_count_limits_monotone_and_continuous_estimate():
     T, H, W, gamma = 21, 45, 80, 0.6
     radii = oracle.default_radii(T, H, W, gamma)
