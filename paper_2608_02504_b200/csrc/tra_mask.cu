@@ -47,14 +47,19 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
                       int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal) {
   extern __shared__ int32_t s_dyn[];
   __shared__ int s_rank_ridx[128];
+  __shared__ uint32_t s_sorted[128];        // queries in descending candidate index: coord | 0, and ...
+  __shared__ uint16_t s_sorted_r[128];      // ... their candidate index
   __shared__ tra_block_boxes_t s_ubox;
   __shared__ int s_rstar, s_count, s_whole;
 
   const int Wp = (W + 1) | 1;                                      // odd row stride
+  const int Tp = (T + 3) & ~3;                                     // keeps s_diff 16-byte aligned
+  const int n_diff = (H * Wp + 3) & ~3;                            // words of the count field, padded to 16 bytes
   int32_t* s_theta_star = s_dyn;                                   // [T]
-  int32_t* s_frame_needed = s_dyn + T;                             // [T]
-  int32_t* s_diff = s_dyn + 2 * T;                                 // [H * (W + 1)]
-  uint16_t* s_ne = (uint16_t*)(s_diff + H * Wp);                   // [NB] reached columns
+  int32_t* s_frame_ylo = s_dyn + Tp;                               // [T] rows of the frame that hold keys of an
+  int32_t* s_frame_yhi = s_dyn + 2 * Tp;                           // [T] undecided key block (yhi < 0: none)
+  int32_t* s_diff = s_dyn + 3 * Tp;                                // [H * (W + 1)]
+  uint16_t* s_ne = (uint16_t*)(s_diff + n_diff);                   // [NB] reached columns
   uint16_t* s_hi = s_ne + NB;                                      // [NB] high columns
   uint8_t* s_state = (uint8_t*)(s_hi + NB);                        // [NB] 0 / 1 decided, 2 undecided
 
@@ -90,14 +95,19 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     s_count = 0;
     s_rstar = -1;
   }
-  for (int i = tid; i < T; i += TRA_MASK_THREADS) s_frame_needed[i] = 0;
+  for (int i = tid; i < T; i += TRA_MASK_THREADS) {
+    s_frame_ylo[i] = H;
+    s_frame_yhi[i] = -1;
+  }
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
     s_ne[v] = 0;
     s_hi[v] = 0;
   }
   __syncthreads();
 
-  // r*: the need-th largest candidate index (ties broken by lane order)
+  // r*: the need-th largest candidate index (ties broken by lane order).  The ranks also re-deal
+  // the queries to the threads in descending candidate order, so that the threads of a warp draw
+  // disks of similar size (the row loops below run as long as the largest disk of the warp).
   if (tid < nq) {
     int rank = 0;
     for (int j = 0; j < nq; ++j) {
@@ -105,8 +115,17 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       rank += (o > qr) || (o == qr && j < tid);
     }
     if (rank == need - 1) s_rstar = qr;
+    s_sorted[rank] = tra_pack_coord(qt, qy, qx);
+    s_sorted_r[rank] = (uint16_t)qr;
   }
   __syncthreads();
+  if (tid < nq) {
+    const uint32_t c = s_sorted[tid];
+    qx = tra_coord_x(c);
+    qy = tra_coord_y(c);
+    qt = tra_coord_t(c);
+    qr = s_sorted_r[tid];
+  }
   const int rstar = s_rstar;                            // -1: fewer than `need` valid queries
   if (rstar >= 0)
     for (int i = tid; i < T; i += TRA_MASK_THREADS) s_theta_star[i] = theta[rstar * T + i];
@@ -140,9 +159,13 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     if (keep_diagonal && v == u) decided = 1;
     s_state[v] = (uint8_t)decided;
     if (decided == 2) {
-      // frames this key block has tokens in
-      int f0 = (v * b) / HW, f1 = (min(N, (v + 1) * b) - 1) / HW;
-      for (int f = f0; f <= f1; ++f) s_frame_needed[f] = 1;
+      // frames this key block has tokens in, and the rows of each that hold them
+      const tra_block_boxes_t vb = boxes[v];
+      for (int iv = 0; iv < vb.n_box; ++iv)
+        for (int f = vb.box[iv].t0; f <= vb.box[iv].t1; ++f) {
+          atomicMin(&s_frame_ylo[f], (int)vb.box[iv].y0);
+          atomicMax(&s_frame_yhi[f], (int)vb.box[iv].y1);
+        }
     } else {
       mask_row[v] = (uint8_t)decided;
       kept += decided;
@@ -153,8 +176,10 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
 
   // ---- 2. count field of every frame that holds an undecided key block ---------------------
   // builds the field for the frame distance dist(thread) -> |f - t_i| of every query
-  auto build_field = [&](auto dist_of_query) {
-    for (int i = tid; i < H * Wp; i += TRA_MASK_THREADS) s_diff[i] = 0;
+  // Only the rows win_lo .. win_hi of the frame are read afterwards: the field is built for them alone.
+  auto build_field = [&](auto dist_of_query, int win_lo, int win_hi) {
+    for (int i = (win_lo * Wp) / 4 + tid; i < ((win_hi + 1) * Wp + 3) / 4; i += TRA_MASK_THREADS)
+      reinterpret_cast<uint4*>(s_diff)[i] = make_uint4(0u, 0u, 0u, 0u);
     if (tid == 0) s_whole = 0;
     __syncthreads();
     if (tid < nq) {
@@ -164,7 +189,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
         atomicAdd(&s_whole, 1);                       // the disk covers the whole frame
       } else {
         const int R = tra_isqrt_small(th);
-        const int ylo = max(0, qy - R), yhi = min(H - 1, qy + R);
+        const int ylo = max(win_lo, qy - R), yhi = min(win_hi, qy + R);
         for (int yy = ylo; yy <= yhi; ++yy) {
           const int dy = yy - qy;
           const int rem = th - dy * dy;
@@ -180,20 +205,29 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       }
     }
     __syncthreads();
-    // prefix sum along x: one thread per row (the row stride W + 1 is made odd, so the threads
-    // of a warp walk different banks)
-    for (int yy = tid; yy < H; yy += TRA_MASK_THREADS) {
-      int32_t* row = s_diff + yy * Wp;
-      int run = 0;
-      for (int x0 = 0; x0 < W; x0 += 8) {          // eight independent loads, then the running sum
-        int v[8];
+    // prefix sum along x: two threads (a lane pair) per row, each over half of it; the second adds
+    // the first one's total (the row stride W + 1 is odd, so the threads of a warp walk different banks)
+    {
+      const int half_w = (W + 1) >> 1;
+      for (int yy0 = win_lo; yy0 <= win_hi; yy0 += TRA_MASK_THREADS / 2) {
+        const int yy = yy0 + (tid >> 1), part = tid & 1;
+        const bool on = yy <= win_hi;
+        int32_t* row = s_diff + (on ? yy : 0) * Wp;
+        const int xa = part ? half_w : 0, xb = part ? W : half_w;
+        int run = 0;
+        for (int x0 = xa; x0 < xb && on; x0 += 8) {   // eight independent loads, then the running sum
+          int v[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = x0 + j < W ? row[x0 + j] : 0;
+          for (int j = 0; j < 8; ++j) v[j] = x0 + j < xb ? row[x0 + j] : 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          run += v[j];
-          if (x0 + j < W) row[x0 + j] = run;
+          for (int j = 0; j < 8; ++j) {
+            run += v[j];
+            if (x0 + j < xb) row[x0 + j] = run;
+          }
         }
+        const int left = __shfl_xor_sync(0xffffffffu, run, 1);       // the other half's total
+        if (on && part)
+          for (int x = xa; x < xb; ++x) row[x] += left;
       }
     }
     __syncthreads();
@@ -207,13 +241,18 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       if (s_state[v] != 2) continue;
       const int ps = max(v * b, p_begin), pe = min((v + 1) * b, p_end);
       int ne = 0, hi = 0;
-      for (int p0 = ps; p0 < pe; p0 += 32) {
-        const int p = p0 + lane;
+      // b <= 128: at most four keys per lane; their coordinate loads are in flight together
+      uint32_t kc[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int p = ps + 32 * i + lane;
+        kc[i] = p < pe ? __ldg(coord_packed + p) : 0xffffffffu;
+      }
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (ps + 32 * i >= pe) break;                     // uniform across the warp
         int c = 0;
-        if (p < pe) {
-          const uint32_t kc = coord_packed[p];
-          c = s_diff[tra_coord_y(kc) * Wp + tra_coord_x(kc)] + whole;
-        }
+        if (kc[i] != 0xffffffffu) c = s_diff[tra_coord_y(kc[i]) * Wp + tra_coord_x(kc[i])] + whole;
         ne += __popc(__ballot_sync(0xffffffffu, c > 0));
         hi += __popc(__ballot_sync(0xffffffffu, 3 * c > b));
       }
@@ -232,18 +271,20 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     const int t0 = s_ubox.box[0].t0;
     for (int k = 0; k < T; ++k) {
       const int fa = t0 - k, fb = t0 + k;
-      const bool need_a = fa >= 0 && s_frame_needed[fa];
-      const bool need_b = k > 0 && fb < T && s_frame_needed[fb];
+      const bool need_a = fa >= 0 && s_frame_yhi[fa] >= 0;
+      const bool need_b = k > 0 && fb < T && s_frame_yhi[fb] >= 0;
       if (!need_a && !need_b) continue;                 // uniform across the CTA
-      build_field([&]() { return k; });
+      const int win_lo = min(need_a ? s_frame_ylo[fa] : H, need_b ? s_frame_ylo[fb] : H);
+      const int win_hi = max(need_a ? s_frame_yhi[fa] : -1, need_b ? s_frame_yhi[fb] : -1);
+      build_field([&]() { return k; }, win_lo, win_hi);
       if (need_a) count_frame(fa);
       if (need_b) count_frame(fb);
       __syncthreads();
     }
   } else {
     for (int f = 0; f < T; ++f) {
-      if (!s_frame_needed[f]) continue;                 // uniform across the CTA
-      build_field([&]() { return abs(qt - f); });
+      if (s_frame_yhi[f] < 0) continue;                 // uniform across the CTA
+      build_field([&]() { return abs(qt - f); }, s_frame_ylo[f], s_frame_yhi[f]);
       count_frame(f);
       __syncthreads();
     }
@@ -440,7 +481,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   const long long rows = BH * NB;
 
   const int H = plan->cfg.H, W = plan->cfg.W;
-  size_t smem = ((size_t)2 * T + (size_t)H * ((W + 1) | 1)) * sizeof(int32_t) + (size_t)NB * 5;
+  size_t smem = ((size_t)3 * ((T + 3) & ~3) + (((size_t)H * ((W + 1) | 1) + 3) & ~(size_t)3)) * sizeof(int32_t) +
+                (size_t)NB * 5;
   smem = (smem + 15) & ~(size_t)15;
   if (smem > 200 * 1024) return TRA_ERR_UNSUPPORTED;     // frame too large for the count field
   dim3 grid((unsigned)NB, (unsigned)BH);
