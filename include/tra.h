@@ -44,6 +44,9 @@ extern "C" {
 #define TRA_ERR_CAPACITY (-3)    /* col_idx capacity too small (reported by tra_plan_status)   */
 #define TRA_ERR_CUDA (-4)        /* a CUDA runtime / driver call failed                        */
 #define TRA_ERR_TIMEOUT (-5)     /* a bounded device-side wait expired (reported by tra_plan_status) */
+#define TRA_ERR_BOUNDS (-6)      /* debug build (-DTRA_DEBUG) only: a kernel computed an index outside its   */
+                                 /* array, or its roles disagree on the work they walked; the access was    */
+                                 /* skipped (reported by tra_plan_status)                                    */
 
 /* plan flags */
 #define TRA_KEEP_DIAGONAL 1u /* force block_mask[u][u] = 1 (a token always sees itself, Eq. 15) */
@@ -99,7 +102,8 @@ int tra_plan_tables(const tra_plan_t* plan, double* radii, int32_t* theta, int32
 int tra_plan_count_table(const tra_plan_t* plan, uint32_t* counts);
 
 /* Reads and clears the plan's device status word (synchronises `stream`): TRA_OK, or the
- * first TRA_ERR_CAPACITY / TRA_ERR_TIMEOUT a kernel of this plan recorded since the last call. */
+ * first TRA_ERR_CAPACITY / TRA_ERR_TIMEOUT / TRA_ERR_BOUNDS a kernel of this plan recorded since the
+ * last call. */
 int tra_plan_status(tra_plan_t* plan, void* stream);
 
 const char* tra_status_string(int status);

@@ -324,6 +324,7 @@ struct SharedCtl {
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
+  int dbg_jobs[4];          // bounds-checking build: jobs walked by softmax tile 0 / tile 1 / the MMA warp, entries loaded
   int rmax[4];              // largest candidate index among the video queries of each query block
   uint32_t bitmap[4][kMaxBitmapWords];
 };
@@ -406,7 +407,10 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   for (int i = tid; i < 4 * kMaxBitmapWords; i += kThreads) (&ctl->bitmap[0][0])[i] = 0u;
-  if (tid < 4) ctl->rmax[tid] = -1;
+  if (tid < 4) {
+    ctl->rmax[tid] = -1;
+    ctl->dbg_jobs[tid] = 0;
+  }
   __syncthreads();
   // Token-mask launch without a block list (Eq. 16 itself): the key blocks a query block can reach
   // at all, from the block boxes and the largest candidate index among its queries — a superset
@@ -426,19 +430,27 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       if (t < 0 || ub >= NB) continue;
       const bool q_text = (ub + 1) * BN > tm.n_video;        // holds a text query: sees every key
       const int rmax = ctl->rmax[g];
-      const tra_block_boxes_t ubx = tm.boxes[ub];
+      const tra_block_boxes_t* ubx = tm.boxes + ub;      // read in place: a local copy indexed by a loop
+      const int n_ubox = ubx->n_box;                    // variable would live in local memory
       for (int v = tid; v < NB; v += kThreads) {
         bool on = q_text || (v + 1) * BN > tm.n_video;         // text keys are always visible
         if (!on && rmax >= 0) {
-          const tra_block_boxes_t vb = tm.boxes[v];
-          for (int iu = 0; iu < ubx.n_box && !on; ++iu)
-            for (int iv = 0; iv < vb.n_box && !on; ++iv) {
-              const tra_box_t a = ubx.box[iu], c = vb.box[iv];
-              const int dt_min = max(0, max(a.t0 - c.t1, c.t0 - a.t1));
-              const int gy = max(0, max(a.y0 - c.y1, c.y0 - a.y1));
-              const int gx = max(0, max(a.x0 - c.x1, c.x0 - a.x1));
+          const tra_block_boxes_t* vb = tm.boxes + v;
+          const int n_vbox = vb->n_box;
+          for (int iu = 0; iu < n_ubox && !on; ++iu) {
+            const uint4 au = __ldg(reinterpret_cast<const uint4*>(&ubx->box[iu]));
+            const int a_t0 = (int16_t)(au.x & 0xffffu), a_t1 = (int16_t)(au.x >> 16), a_y0 = (int16_t)(au.y & 0xffffu),
+                      a_y1 = (int16_t)(au.y >> 16), a_x0 = (int16_t)(au.z & 0xffffu), a_x1 = (int16_t)(au.z >> 16);
+            for (int iv = 0; iv < n_vbox && !on; ++iv) {
+              const uint4 cu = __ldg(reinterpret_cast<const uint4*>(&vb->box[iv]));
+              const int c_t0 = (int16_t)(cu.x & 0xffffu), c_t1 = (int16_t)(cu.x >> 16), c_y0 = (int16_t)(cu.y & 0xffffu),
+                        c_y1 = (int16_t)(cu.y >> 16), c_x0 = (int16_t)(cu.z & 0xffffu), c_x1 = (int16_t)(cu.z >> 16);
+              const int dt_min = max(0, max(a_t0 - c_t1, c_t0 - a_t1));
+              const int gy = max(0, max(a_y0 - c_y1, c_y0 - a_y1));
+              const int gx = max(0, max(a_x0 - c_x1, c_x0 - a_x1));
               on = tm.theta[rmax * tm.T + dt_min] >= gy * gy + gx * gx;
             }
+          }
         }
         if (on) atomicOr(&ctl->bitmap[g][v >> 5], 1u << (v & 31));
       }
@@ -452,6 +464,10 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     {
       const long long r = (long long)bh * NB + ub;
       const int lo = row_ptr[r], hi = row_ptr[r + 1];
+#ifdef TRA_DEBUG      // the list of a row lies inside the lists of the launch
+      if (tid == 0 && (lo < 0 || hi < lo || hi > row_ptr[(long long)gridDim.y * NB]))
+        tra_set_status(status, TRA_ERR_BOUNDS);
+#endif
       for (int e = lo + tid; e < hi; e += kThreads) {
         const int v = col_idx[e];
         if (v >= 0 && v < NB) atomicOr(&ctl->bitmap[g][v >> 5], 1u << (v & 31));
@@ -578,6 +594,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
             ++seen;
           }
         }
+#ifdef TRA_DEBUG
+        ctl->dbg_jobs[3] = (int)ks.jobs - (ks.e == vs.e ? 0 : 1 << 20);     // both streams walked every entry
+#endif
       }
     }
   } else if (warp == 9) {
@@ -790,6 +809,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           tc_commit(smem_u32(&ctl->kv_release[(n + 1u) & 15u]));   // commit n + 1 of the release sequence
           cur = nxt;
           nxt = ahead;
+#ifdef TRA_DEBUG
+          if (lane == 0) ctl->dbg_jobs[2] = (int)n + 1;
+#endif
         }
       }
       // make sure every MMA has retired before tensor memory is released
@@ -888,30 +910,27 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const uint4* kc4 = reinterpret_cast<const uint4*>(tm.coord_packed + k0);
           const bool one_frame = k0 + BN <= tm.n_video && tra_coord_t(tm.coord_packed[k0 + BN - 1]) == kt0;
           // 16-key slices of the block; the usual case: each is 16 consecutive x of one frame row
-          uint32_t sl[BN / 16];
-#pragma unroll
-          for (int q = 0; q < BN / 64; ++q) {
-            const uint4 w4 = __ldg(reinterpret_cast<const uint4*>(tm.slice + (k0 >> 4)) + q);
-            sl[4 * q] = w4.x;
-            sl[4 * q + 1] = w4.y;
-            sl[4 * q + 2] = w4.z;
-            sl[4 * q + 3] = w4.w;
-          }
-          uint32_t all_runs = sl[0];
-#pragma unroll
-          for (int q = 1; q < BN / 16; ++q) all_runs &= sl[q];
+          const uint4 sa = __ldg(reinterpret_cast<const uint4*>(tm.slice + (k0 >> 4)));
+          const uint4 sb4 = BN > 64 ? __ldg(reinterpret_cast<const uint4*>(tm.slice + (k0 >> 4)) + 1) : sa;
+          auto slice_word = [&](int q) -> uint32_t {     // q is a compile-time constant at every use
+            const uint4& w4 = q < 4 ? sa : sb4;
+            return (q & 3) == 0 ? w4.x : ((q & 3) == 1 ? w4.y : ((q & 3) == 2 ? w4.z : w4.w));
+          };
+          const uint32_t all_runs = sa.x & sa.y & sa.z & sa.w & sb4.x & sb4.y & sb4.z & sb4.w;
           if (all_runs & (1u << 30)) {
             // A key (x0 + j, ys) is inside the disk iff |x0 + j - qx| <= w with
             // w = floor(sqrt(theta - (ys - qy)^2)): one square root per slice, then an unsigned
             // range test per key:  0 <= j + (x0 - qx + w) <= 2 w.
 #pragma unroll
             for (int q = 0; q < BN / 16; ++q) {
-              const int ts = (int)((sl[q] >> 20) & 1023u), dts = ts - kt0;
-              const int th = dts == 0 ? th0 : (dts == 1 ? th1 : __ldg(th_row + abs(qt - ts)));
-              const int dy = tra_coord_y(sl[q]) - qy;
+              const uint32_t sw = slice_word(q);
+              const int ts = (int)((sw >> 20) & 1023u), dts = ts - kt0;
+              const int th = dts == 0 ? th0
+                             : (dts == 1 ? th1 : (TRA_IDX(abs(qt - ts), tm.T, status) ? __ldg(th_row + abs(qt - ts)) : 0));
+              const int dy = tra_coord_y(sw) - qy;
               const int rem = th - dy * dy;
               const int w = tra_isqrt_small_nocvt(max(rem, 0));
-              const uint32_t base = rem < 0 ? 0x40000000u : (uint32_t)(w + tra_coord_x(sl[q]) - qx);
+              const uint32_t base = rem < 0 ? 0x40000000u : (uint32_t)(w + tra_coord_x(sw) - qx);
               const uint32_t span = (uint32_t)(2 * w);
 #pragma unroll
               for (int j = 0; j < 16; ++j)
@@ -921,10 +940,10 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
             for (int j4 = 0; j4 < BN / 4; ++j4) {
               const uint4 c4 = __ldg(kc4 + j4);
-              const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
               for (int q4 = 0; q4 < 4; ++q4) {
-                const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
+                const uint32_t kc = q4 == 0 ? c4.x : (q4 == 1 ? c4.y : (q4 == 2 ? c4.z : c4.w));
+                const int dx = qx - tra_coord_x(kc), dy = qy - tra_coord_y(kc);
                 if (dx * dx + dy * dy > th0) sb[j4 * 4 + q4] = __float_as_uint(-1e30f);
               }
             }
@@ -932,13 +951,15 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
 #pragma unroll
             for (int j4 = 0; j4 < BN / 4; ++j4) {
               const uint4 c4 = __ldg(kc4 + j4);
-              const uint32_t cs[4] = {c4.x, c4.y, c4.z, c4.w};
 #pragma unroll
               for (int q4 = 0; q4 < 4; ++q4) {
                 const int j = j4 * 4 + q4;
-                const int dt = tra_coord_t(cs[q4]) - kt0;
-                const int th = dt == 0 ? th0 : (dt == 1 ? th1 : __ldg(th_row + abs(qt - kt0 - dt)));
-                const int dx = qx - tra_coord_x(cs[q4]), dy = qy - tra_coord_y(cs[q4]);
+                const uint32_t kc = q4 == 0 ? c4.x : (q4 == 1 ? c4.y : (q4 == 2 ? c4.z : c4.w));
+                const int dt = tra_coord_t(kc) - kt0;
+                const int th = dt == 0 ? th0
+                               : (dt == 1 ? th1
+                                          : (TRA_IDX(abs(qt - kt0 - dt), tm.T, status) ? __ldg(th_row + abs(qt - kt0 - dt)) : 0));
+                const int dx = qx - tra_coord_x(kc), dy = qy - tra_coord_y(kc);
                 if (k0 + j < tm.n_video && dx * dx + dy * dy > th) sb[j] = __float_as_uint(-1e30f);
               }
             }
@@ -1049,6 +1070,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       jobs_before += __popc(word0) + __popc(word1);
     }
 
+#ifdef TRA_DEBUG
+    if (r == 0) ctl->dbg_jobs[k] = (int)n;
+#endif
     // ---- epilogue: O = o / l, entropy, lse ------------------------------------------------
     // the MMA warp commits `drain` behind its last MMA: every PV of both tiles has retired then
     if (alive && n > 0)
@@ -1095,6 +1119,11 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // ---- teardown ------------------------------------------------------------------------
   tc_fence_before();
   __syncthreads();
+#ifdef TRA_DEBUG      // every role walked the same job stream (block-sparse launches)
+  if (!kDense && tid == 0 && !ctl->abort_flag &&
+      (ctl->dbg_jobs[0] + ctl->dbg_jobs[1] != ctl->dbg_jobs[2] || ctl->dbg_jobs[3] != ctl->dbg_jobs[2]))
+    tra_set_status(status, TRA_ERR_BOUNDS);
+#endif
   if (warp == 9) {
     if (ctl->abort_flag) {
       // let copies and MMAs that were in flight when the CTA gave up land before releasing

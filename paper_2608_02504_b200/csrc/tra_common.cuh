@@ -41,6 +41,7 @@ struct tra_plan {
   int32_t* d_theta;               // [n_radii][T]
   float* d_radii_f32;             // [n_radii]
   uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)
+  uint32_t* d_counts_coarse;      // [T*H*W][16] every eighth entry of a row (n_radii <= 128), else NULL
   tra_block_boxes_t* d_boxes;     // [NB]
   int* d_status;                  // device status word
   // copy streams of tra_hot_path_host, created on its first call with this plan
@@ -60,5 +61,23 @@ __host__ __device__ inline int tra_coord_t(uint32_t c) { return (int)(c >> 20); 
     if (_e != cudaSuccess) return TRA_ERR_CUDA;   \
   } while (0)
 
+// Plan time: the coarse table of the two-round radius search (tra_radius.cu).
+int tra_build_coarse_table(const uint32_t* counts, uint32_t* coarse, long long cells, int n_radii, int* status,
+                           cudaStream_t stream);
+
 // Records the first error code in the plan's device status word.
 __device__ inline void tra_set_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+// Bounds-checking build (-DTRA_DEBUG): TRA_IDX(i, n, status) is true when 0 <= i < n; otherwise it
+// records TRA_ERR_BOUNDS and the caller skips the access.  In the normal build it is the constant
+// true and the guarded access compiles to the plain one.
+#ifdef TRA_DEBUG
+__device__ inline bool tra_index_ok(long long i, long long n, int* status) {
+  if (i >= 0 && i < n) return true;
+  tra_set_status(status, TRA_ERR_BOUNDS);
+  return false;
+}
+#define TRA_IDX(i, n, status) tra_index_ok((long long)(i), (long long)(n), (status))
+#else
+#define TRA_IDX(i, n, status) true
+#endif

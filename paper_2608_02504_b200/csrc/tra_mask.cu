@@ -44,7 +44,8 @@ __global__ void __launch_bounds__(TRA_MASK_THREADS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
                       uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int S, int NB,
-                      int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal) {
+                      int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal,
+                      int* __restrict__ status) {
   extern __shared__ int32_t s_dyn[];
   __shared__ int s_rank_ridx[128];
   __shared__ uint32_t s_sorted[128];        // queries in descending candidate index: coord | 0, and ...
@@ -82,7 +83,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
 
   // this thread's query
   int qx = 0, qy = 0, qt = 0, qr = 0;
-  if (tid < nq) {
+  if (tid < nq && TRA_IDX(q0 + tid, N, status)) {
     uint32_t c = coord_packed[q0 + tid];
     qx = tra_coord_x(c);
     qy = tra_coord_y(c);
@@ -90,6 +91,9 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     qr = min((int)ridx_h[q0 + tid], n_radii - 1);      // a candidate index past the table reads its last row
     s_rank_ridx[tid] = qr;
   }
+#ifdef TRA_DEBUG
+  if (tid < nq && (qx >= W || qy >= H || qt >= T)) tra_set_status(status, TRA_ERR_BOUNDS);   // indexes the count field
+#endif
   if (tid == 0) {
     s_ubox = boxes[u];
     s_count = 0;
@@ -115,8 +119,10 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       rank += (o > qr) || (o == qr && j < tid);
     }
     if (rank == need - 1) s_rstar = qr;
-    s_sorted[rank] = tra_pack_coord(qt, qy, qx);
-    s_sorted_r[rank] = (uint16_t)qr;
+    if (TRA_IDX(rank, nq, status)) {
+      s_sorted[rank] = tra_pack_coord(qt, qy, qx);
+      s_sorted_r[rank] = (uint16_t)qr;
+    }
   }
   __syncthreads();
   if (tid < nq) {
@@ -150,6 +156,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
           int gx = max(0, max(a.x0 - c.x1, c.x0 - a.x1));
           int fy = max(a.y1 - c.y0, c.y1 - a.y0);
           int fx = max(a.x1 - c.x0, c.x1 - a.x0);
+          if (!TRA_IDX(dt_max, T, status)) continue;       // dt_min <= dt_max
           if (s_theta_star[dt_min] >= gy * gy + gx * gx) all_reject = false;
           if (s_theta_star[dt_max] < fy * fy + fx * fx) all_accept = false;
         }
@@ -163,6 +170,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       const tra_block_boxes_t vb = boxes[v];
       for (int iv = 0; iv < vb.n_box; ++iv)
         for (int f = vb.box[iv].t0; f <= vb.box[iv].t1; ++f) {
+          if (!TRA_IDX(f, T, status)) break;
           atomicMin(&s_frame_ylo[f], (int)vb.box[iv].y0);
           atomicMax(&s_frame_yhi[f], (int)vb.box[iv].y1);
         }
@@ -199,6 +207,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
             lo = max(0, qx - w);
             hi = min(W - 1, qx + w) + 1;
           }
+          if (!TRA_IDX(yy * Wp + hi, H * Wp, status)) continue;      // lo <= hi <= W < Wp
           atomicAdd(&s_diff[yy * Wp + lo], 1);
           atomicAdd(&s_diff[yy * Wp + hi], -1);
         }
@@ -252,7 +261,8 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       for (int i = 0; i < 4; ++i) {
         if (ps + 32 * i >= pe) break;                     // uniform across the warp
         int c = 0;
-        if (kc[i] != 0xffffffffu) c = s_diff[tra_coord_y(kc[i]) * Wp + tra_coord_x(kc[i])] + whole;
+        if (kc[i] != 0xffffffffu && TRA_IDX(tra_coord_y(kc[i]) * Wp + tra_coord_x(kc[i]), H * Wp, status))
+          c = s_diff[tra_coord_y(kc[i]) * Wp + tra_coord_x(kc[i])] + whole;
         ne += __popc(__ballot_sync(0xffffffffu, c > 0));
         hi += __popc(__ballot_sync(0xffffffffu, 3 * c > b));
       }
@@ -274,8 +284,9 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       const bool need_a = fa >= 0 && s_frame_yhi[fa] >= 0;
       const bool need_b = k > 0 && fb < T && s_frame_yhi[fb] >= 0;
       if (!need_a && !need_b) continue;                 // uniform across the CTA
-      const int win_lo = min(need_a ? s_frame_ylo[fa] : H, need_b ? s_frame_ylo[fb] : H);
-      const int win_hi = max(need_a ? s_frame_yhi[fa] : -1, need_b ? s_frame_yhi[fb] : -1);
+      int win_lo = min(need_a ? s_frame_ylo[fa] : H, need_b ? s_frame_ylo[fb] : H);
+      int win_hi = max(need_a ? s_frame_yhi[fa] : -1, need_b ? s_frame_yhi[fb] : -1);
+      if (!TRA_IDX(win_lo, H, status) || !TRA_IDX(win_hi, H, status)) win_lo = 0, win_hi = H - 1;
       build_field([&]() { return k; }, win_lo, win_hi);
       if (need_a) count_frame(fa);
       if (need_b) count_frame(fb);
@@ -346,7 +357,8 @@ tra_row_ptr_scan_kernel(int32_t* __restrict__ row_ptr, long long rows, long long
 // ---------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* __restrict__ row_ptr,
-                        int32_t* __restrict__ col_idx, long long rows, int NB, long long capacity) {
+                        int32_t* __restrict__ col_idx, long long rows, int NB, long long capacity,
+                        int* __restrict__ status) {
   const int lane = threadIdx.x & 31;
   const long long row = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   if (row >= rows) return;
@@ -358,7 +370,7 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
     unsigned bal = __ballot_sync(0xffffffffu, keep);
     if (keep) {
       long long pos = base + __popc(bal & ((1u << lane) - 1u));
-      if (pos < capacity) col_idx[pos] = v;
+      if (pos < capacity && TRA_IDX(pos, capacity, status)) col_idx[pos] = v;
     }
     base += __popc(bal);
   }
@@ -383,7 +395,8 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 #define TRA_PAIR_THREADS 256
 
 __global__ void __launch_bounds__(TRA_PAIR_THREADS)
-tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restrict__ pairs, int NB, int NT, int G) {
+tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restrict__ pairs, int NB, int NT, int G,
+                      int* __restrict__ status) {
   extern __shared__ uint32_t s_pair[];
   const int words = (NB + 31) >> 5;
   const int win_rows = TRA_PAIR_CHUNK + TRA_PAIR_WINDOW;
@@ -457,7 +470,7 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
         if (free_mask) v = base + __ffs(free_mask) - 1;
       }
     }
-    if (lane == 0) {
+    if (lane == 0 && TRA_IDX(n_out, (NT + 1) / 2, status) && (v == -1 || TRA_IDX(v, NT, status))) {
       s_used[u] = 1;
       if (v >= 0) s_used[v] = 1;
       out[2 * n_out] = u;
@@ -491,13 +504,14 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
                                         (int)smem));
   tra_block_vote_kernel<<<grid, TRA_MASK_THREADS, smem, stream>>>(
       ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, plan->S, NB,
-      plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0);
+      plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0,
+      plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,
                                                   plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_col_idx_fill_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(
-      block_mask, row_ptr, col_idx, rows, NB, (long long)col_idx_capacity);
+      block_mask, row_ptr, col_idx, rows, NB, (long long)col_idx_capacity, plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   if (tile_pairs) {
     // query tiles of the attention launch: 128 rows = G blocks (block sizes that do not divide 128
@@ -511,7 +525,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     if (pair_smem > 48 * 1024)
       TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)pair_smem));
-    tra_pair_tiles_kernel<<<(unsigned)BH, TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G);
+    tra_pair_tiles_kernel<<<(unsigned)BH, TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G,
+                                                                                 plan->d_status);
     TRA_CUDA_CHECK(cudaGetLastError());
   }
   return TRA_OK;

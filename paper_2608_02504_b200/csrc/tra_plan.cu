@@ -36,7 +36,7 @@ __device__ __forceinline__ uint32_t tra_frame_count(int y, int x, int H, int W, 
 
 __global__ void tra_count_table_kernel(int T, int H, int W, int n_radii,
                                        const int32_t* __restrict__ theta,
-                                       uint32_t* __restrict__ counts) {
+                                       uint32_t* __restrict__ counts, int* __restrict__ status) {
   int g = blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= H * W * n_radii) return;
   int k = g % n_radii;
@@ -47,11 +47,13 @@ __global__ void tra_count_table_kernel(int T, int H, int W, int n_radii,
   for (int delta = 0; delta < T; ++delta) c += tra_frame_count(y, x, H, W, th[delta]);
   size_t frame_stride = (size_t)H * W * n_radii;
   size_t base = (size_t)yx * n_radii + k;
-  counts[base] = c;  // f = 0
+  const size_t n_counts = frame_stride * T;
+  if (TRA_IDX(base, n_counts, status)) counts[base] = c;  // f = 0
   for (int f = 0; f + 1 < T; ++f) {
     c += tra_frame_count(y, x, H, W, th[f + 1]);
     c -= tra_frame_count(y, x, H, W, th[T - 1 - f]);
-    counts[base + (size_t)(f + 1) * frame_stride] = c;
+    if (TRA_IDX(base + (size_t)(f + 1) * frame_stride, n_counts, status))
+      counts[base + (size_t)(f + 1) * frame_stride] = c;
   }
 }
 
@@ -61,7 +63,8 @@ __global__ void tra_count_table_kernel(int T, int H, int W, int n_radii,
 template <bool kGather>
 __global__ void tra_permute_rows_kernel(const int32_t* __restrict__ raster_of_pos,
                                         const uint4* __restrict__ src, uint4* __restrict__ dst,
-                                        int N, int S, int chunks_per_row, long long total_chunks) {
+                                        int N, int S, int chunks_per_row, long long total_chunks,
+                                        int* __restrict__ status) {
   long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= total_chunks) return;
   int chunk = (int)(g % chunks_per_row);
@@ -69,6 +72,7 @@ __global__ void tra_permute_rows_kernel(const int32_t* __restrict__ raster_of_po
   int p = (int)(row % S);
   long long bh = row / S;
   long long other = bh * S + (p < N ? raster_of_pos[p] : p);   // text tokens stay in place
+  if (!TRA_IDX(other * chunks_per_row + chunk, total_chunks, status)) return;
   if (kGather)
     dst[row * chunks_per_row + chunk] = src[other * chunks_per_row + chunk];
   else
@@ -101,6 +105,7 @@ static void tra_plan_free(tra_plan* p) {
   cudaFree(p->d_theta);
   cudaFree(p->d_radii_f32);
   cudaFree(p->d_counts);
+  cudaFree(p->d_counts_coarse);
   cudaFree(p->d_boxes);
   cudaFree(p->d_status);
   if (p->copy_in) cudaStreamDestroy(p->copy_in);
@@ -268,6 +273,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
             cudaMalloc(&p->d_theta, sizeof(int32_t) * nr * T) == cudaSuccess &&
             cudaMalloc(&p->d_radii_f32, sizeof(float) * nr) == cudaSuccess &&
             cudaMalloc(&p->d_counts, sizeof(uint32_t) * count_elems) == cudaSuccess &&
+            (nr > 128 || cudaMalloc(&p->d_counts_coarse, sizeof(uint32_t) * 16 * (size_t)p->N) == cudaSuccess) &&
             cudaMalloc(&p->d_boxes, sizeof(tra_block_boxes_t) * p->NB) == cudaSuccess &&
             cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess;
   ok = ok &&
@@ -287,8 +293,11 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   if (ok) {
     int total = H * W * nr;
     tra_count_table_kernel<<<(total + 127) / 128, 128, 0, stream>>>(T, H, W, nr, p->d_theta,
-                                                                    p->d_counts);
-    ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(stream) == cudaSuccess;
+                                                                    p->d_counts, p->d_status);
+    ok = cudaGetLastError() == cudaSuccess;
+    if (ok && p->d_counts_coarse)
+      ok = tra_build_coarse_table(p->d_counts, p->d_counts_coarse, (long long)p->N, nr, p->d_status, stream) == TRA_OK;
+    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
   }
   if (!ok) {
     tra_plan_free(p);
@@ -342,6 +351,7 @@ extern "C" const char* tra_status_string(int status) {
     case TRA_ERR_CAPACITY: return "col_idx capacity too small";
     case TRA_ERR_CUDA: return "CUDA call failed";
     case TRA_ERR_TIMEOUT: return "bounded device-side wait expired";
+    case TRA_ERR_BOUNDS: return "debug build: index out of range or inconsistent work lists";
     default: return "unknown status";
   }
 }
@@ -357,10 +367,10 @@ static int tra_permute(const tra_plan_t* plan, const void* src, void* dst, int n
   if (grid > 0x7fffffffll) return TRA_ERR_UNSUPPORTED;
   if (gather)
     tra_permute_rows_kernel<true><<<(unsigned)grid, 256, 0, stream>>>(
-        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, plan->S, chunks, total);
+        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, plan->S, chunks, total, plan->d_status);
   else
     tra_permute_rows_kernel<false><<<(unsigned)grid, 256, 0, stream>>>(
-        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, plan->S, chunks, total);
+        plan->d_raster_of_pos, (const uint4*)src, (uint4*)dst, plan->N, plan->S, chunks, total, plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }
