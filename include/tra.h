@@ -18,10 +18,12 @@
  *
  * Joint text-video attention (Section 3.2, last paragraph; Algorithm 1).  With cfg.n_text > 0 a
  * sequence is the N video tokens followed by n_text text tokens, S = N + n_text; S takes the place
- * of N in every shape below and NB = ceil(S / block).  The first B_v = ceil(N / block) blocks are
- * video blocks; a block pair with u >= B_v or v >= B_v is always kept, video blocks vote over their
- * video tokens only, the gather/scatter leaves text tokens where they are, and text positions get
- * budget S, radius +inf and the last candidate index.
+ * of N in every shape below and NB = ceil(S / block).  The first B_v = floor(N / block) blocks, made
+ * of video tokens only, are the video blocks; a block pair with u >= B_v or v >= B_v is always kept
+ * (this includes the block that holds both the last video and the first text tokens, so that every
+ * text key stays visible to every query and a text query sees every key), the gather/scatter leaves
+ * text tokens where they are, and text positions get budget S, radius +inf and the last candidate
+ * index.  Without text the ragged last block is a video block like any other.
  *
  * Shapes.  Q, K, V, O: bf16 [B, heads, N, head_dim].  entropy, budget, radius,
  * ridx: [B, heads, N].  block_mask: uint8 [B, heads, NB, NB].  row_ptr: int32
@@ -204,12 +206,16 @@ int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const 
  * memory is needed for the copies to overlap; pageable memory works but serialises.
  *   workspace : DEVICE memory, 256-byte aligned, at least tra_hot_path_host_workspace_bytes(plan,
  *               group) bytes; owned by the caller, free to reuse once `stream` has passed the call.
- * The call allocates no device memory (it creates the plan's two copy streams on its first use and
- * short-lived events).  It returns after enqueueing; `stream` completes after the last copy in
+ * The call allocates no device memory (on its first uses it creates the plan's two copy streams and
+ * a pool of events, which later calls reuse).  The current device must be the one the plan was
+ * created on.  It returns after enqueueing; `stream` completes after the last copy in
  * either direction, so synchronising `stream` (or an event recorded on it) makes O_host valid.
  * Calls that share a plan or a workspace must be ordered on `stream`.
- * Errors: TRA_ERR_INVALID_ARG (NULL / misaligned pointer, non-positive count or scale),
- * TRA_ERR_CAPACITY (workspace too small), TRA_ERR_CUDA; kernel-side errors as for the four calls. */
+ * Errors: TRA_ERR_INVALID_ARG (NULL / misaligned pointer, non-positive count or scale, another
+ * current device), TRA_ERR_CAPACITY (workspace too small), TRA_ERR_CUDA; kernel-side errors as for
+ * the four calls.  After a non-OK return part of the pass may already be enqueued, with the copy
+ * streams and `stream` waiting on one another: synchronise `stream` before the workspace or the
+ * host buffers are reused. */
 size_t tra_hot_path_host_workspace_bytes(const tra_plan_t* plan, int group);
 int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const void* K_host, const void* V_host,
                       void* O_host, void* workspace, size_t workspace_bytes, int heads, int group,

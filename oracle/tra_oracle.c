@@ -67,8 +67,9 @@ int tra_oracle_tile_major(int T, int H, int W, int tile_h, int tile_w, int32_t* 
 }
 
 /* ------------------------------------------------------------------------- *
- * Candidate radii (Eq. 14: "all candidate radii on the latent grid and a
- * full-support radius").  The paper does not list them; reading taken:
+ * Candidate radii: the set R of Eq. 14, which the paper describes only as the
+ * radii available on the latent grid plus one that reaches full support, without
+ * listing them; reading taken:
  *   policy 0 ("extended"): 0,1,...,D with D = ceil(frame diagonal), then
  *       D*exp(gamma*m) for m = 1..T-1; the last one covers the diagonal even
  *       at the largest frame distance, so it is the full-support radius.
@@ -273,12 +274,15 @@ void tra_oracle_block_vote(const int32_t* coord, int N, int T, int b, const int3
                            const uint16_t* ridx_head, const int32_t* u_list, int n_u,
                            int keep_diagonal, int n_text, uint8_t* out) {
   /* Joint text-video attention (Section 3.2, last paragraph; Algorithm 1): the sequence holds the
-   * N video tokens followed by n_text text tokens, S = N + n_text, NB = ceil(S / b) blocks of which
-   * the first B_v = ceil(N / b) are video blocks.  A pair with u >= B_v or v >= B_v is kept
-   * ("text or non-video blocks remain dense"); video blocks vote over their video tokens only
-   * (q < N, k < N), which is also what happens to the block that straddles the boundary. */
+   * N video tokens followed by n_text text tokens, S = N + n_text, NB = ceil(S / b) blocks.  With
+   * text present the video blocks are the first B_v = floor(N / b) blocks, the ones made of video
+   * tokens only; a pair with u >= B_v or v >= B_v is kept (Algorithm 1 leaves non-video blocks
+   * dense).  The block that holds the last video tokens and the first text tokens counts as
+   * non-video: Section 3.2 keeps every text key visible to every query and lets a text query see
+   * every key, which a vote over that block's video tokens could break.  Without text the ragged
+   * last block is a video block like any other (q < N, k < N). */
   int NB = (N + n_text + b - 1) / b;
-  int NBv = (N + b - 1) / b;
+  int NBv = n_text > 0 ? N / b : (N + b - 1) / b;
 #pragma omp parallel for schedule(dynamic, 1)
   for (int iu = 0; iu < n_u; ++iu) {
     int u = u_list[iu];
@@ -370,58 +374,82 @@ void tra_oracle_attention_rows(const uint16_t* Q, const uint16_t* K, const uint1
 }
 
 /* ------------------------------------------------------------------------- *
- * Algorithm 2 taken step by step in fp64: keys are visited in tiles of
- * `tile` columns; each tile yields (m_r, l_r, a_r, o_r), merged into the
- * running (m, l, a, o) with u = exp(m - m'), v = exp(m_r - m'); at the end
- * O = o / l and H = log l + m - a / l.  All keys visible (dense warm-up pass).
+ * The online form of Algorithm 2 in fp64, written as a merge of partial
+ * softmax states.  A state summarises a set of keys for one query by
+ *   ref  a reference score (the largest score of the set),
+ *   mass = sum exp(s - ref),   smass = sum exp(s - ref) s,
+ *   acc  = sum exp(s - ref) v   (a vector of d values).
+ * Two states of disjoint key sets merge by moving both to the larger reference
+ * (every sum is multiplied by exp(old ref - new ref)) and adding.  The keys are
+ * cut into tiles of `tile` columns, each tile's state is formed on its own and
+ * merged into the running one, as the algorithm's block loop does; at the end
+ * O = acc / mass and H = log mass + ref - smass / mass.  All keys visible (the
+ * dense warm-up pass).  The result does not depend on `tile` beyond rounding.
  * ------------------------------------------------------------------------- */
+typedef struct {
+  double ref, mass, smass;
+  double* acc;
+} softmax_state;
+
+static void state_clear(softmax_state* st, int d) {
+  st->ref = -INFINITY;
+  st->mass = 0.0;
+  st->smass = 0.0;
+  for (int c = 0; c < d; ++c) st->acc[c] = 0.0;
+}
+
+/* into <- into merged with part */
+static void state_merge(softmax_state* into, const softmax_state* part, int d) {
+  double ref = into->ref > part->ref ? into->ref : part->ref;
+  if (ref == -INFINITY) return;                        /* both empty */
+  double f_into = exp(into->ref - ref), f_part = exp(part->ref - ref);   /* exp(-inf) = 0 for an empty side */
+  into->mass = f_into * into->mass + f_part * part->mass;
+  into->smass = f_into * into->smass + f_part * part->smass;
+  for (int c = 0; c < d; ++c) into->acc[c] = f_into * into->acc[c] + f_part * part->acc[c];
+  into->ref = ref;
+}
+
 void tra_oracle_attention_rows_alg2(const uint16_t* Q, const uint16_t* K, const uint16_t* V,
                                     int N, int d, double scale, int tile, const int32_t* rows,
                                     int n_rows, double* O, double* H) {
 #pragma omp parallel
   {
     double* q = (double*)malloc((size_t)d * sizeof(double));
-    double* o = (double*)malloc((size_t)d * sizeof(double));
-    double* o_r = (double*)malloc((size_t)d * sizeof(double));
     double* s = (double*)malloc((size_t)tile * sizeof(double));
+    softmax_state run, part;
+    run.acc = (double*)malloc((size_t)d * sizeof(double));
+    part.acc = (double*)malloc((size_t)d * sizeof(double));
 #pragma omp for schedule(dynamic, 1)
     for (int r = 0; r < n_rows; ++r) {
       int qi = rows[r];
       for (int c = 0; c < d; ++c) q[c] = bf16_widen(Q[(size_t)qi * d + c]);
-      double m = -INFINITY, l = 0.0, a = 0.0;
-      for (int c = 0; c < d; ++c) o[c] = 0.0;
+      state_clear(&run, d);
       for (int j0 = 0; j0 < N; j0 += tile) {
         int w = N - j0 < tile ? N - j0 : tile;
-        double m_r = -INFINITY;
+        /* the state of this tile alone */
+        state_clear(&part, d);
         for (int j = 0; j < w; ++j) {
           double dot = 0.0;
           for (int c = 0; c < d; ++c) dot += q[c] * bf16_widen(K[(size_t)(j0 + j) * d + c]);
           s[j] = scale * dot;
-          if (s[j] > m_r) m_r = s[j];
+          if (s[j] > part.ref) part.ref = s[j];
         }
-        double l_r = 0.0, a_r = 0.0;
-        for (int c = 0; c < d; ++c) o_r[c] = 0.0;
         for (int j = 0; j < w; ++j) {
-          double wj = exp(s[j] - m_r);
-          l_r += wj;
-          a_r += wj * s[j];
-          for (int c = 0; c < d; ++c) o_r[c] += wj * bf16_widen(V[(size_t)(j0 + j) * d + c]);
+          double e = exp(s[j] - part.ref);
+          part.mass += e;
+          part.smass += e * s[j];
+          for (int c = 0; c < d; ++c) part.acc[c] += e * bf16_widen(V[(size_t)(j0 + j) * d + c]);
         }
-        double m_new = m > m_r ? m : m_r;
-        double u = exp(m - m_new), v = exp(m_r - m_new);
-        l = u * l + v * l_r;
-        a = u * a + v * a_r;
-        for (int c = 0; c < d; ++c) o[c] = u * o[c] + v * o_r[c];
-        m = m_new;
+        state_merge(&run, &part, d);
       }
       if (O)
-        for (int c = 0; c < d; ++c) O[(size_t)r * d + c] = o[c] / l;
-      if (H) H[r] = log(l) + m - a / l;
+        for (int c = 0; c < d; ++c) O[(size_t)r * d + c] = run.acc[c] / run.mass;
+      if (H) H[r] = log(run.mass) + run.ref - run.smass / run.mass;
     }
     free(q);
-    free(o);
-    free(o_r);
     free(s);
+    free(run.acc);
+    free(part.acc);
   }
 }
 

@@ -25,7 +25,7 @@ static_assert(sizeof(tra_block_boxes_t) == 80, "block boxes");
 struct tra_plan {
   tra_config_t cfg;
   int N, NB, n_radii;   // N = T*H*W video tokens; NB = blocks of the whole sequence
-  int S, NBv;           // S = N + n_text tokens in the sequence; NBv = ceil(N / block) video blocks
+  int S, NBv;           // S = N + n_text tokens in the sequence; NBv = video blocks (see tra_plan_create)
   int device;
   double z_tau;       // Phi^-1(tau), for the lognormal budget map
   // host copies
@@ -44,8 +44,10 @@ struct tra_plan {
   uint32_t* d_counts_coarse;      // [T*H*W][16] every eighth entry of a row (n_radii <= 128), else NULL
   tra_block_boxes_t* d_boxes;     // [NB]
   int* d_status;                  // device status word
-  // copy streams of tra_hot_path_host, created on its first call with this plan
+  // copy streams and events of tra_hot_path_host, created on its first calls with this plan and kept
   cudaStream_t copy_in, copy_out;
+  cudaEvent_t* events;
+  int n_events;
 };
 
 __host__ __device__ inline uint32_t tra_pack_coord(int t, int y, int x) {

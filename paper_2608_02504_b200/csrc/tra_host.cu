@@ -2,6 +2,8 @@
 // overlap the kernels of the neighbouring groups.  Heads are independent problems (Algorithm 1
 // runs per head, Algorithm 2 per query row), so the pass can be cut anywhere between heads.
 // Only copies, events and calls of the library's own entry points live here.
+#include <stdlib.h>
+
 #include <algorithm>
 #include <vector>
 
@@ -46,16 +48,24 @@ HostPassLayout make_layout(const tra_plan_t* plan, int group) {
   return L;
 }
 
-struct EventPool {   // events of one call; destroyed on return (CUDA releases them once they complete)
-  std::vector<cudaEvent_t> ev;
-  ~EventPool() {
-    for (cudaEvent_t e : ev) cudaEventDestroy(e);
-  }
+// Events of one call, drawn from a pool the plan keeps (created on first use, reused by later
+// calls: recording an event again does not disturb waits that were enqueued on its earlier record).
+struct EventPool {
+  tra_plan_t* plan;
+  int next = 0;
   cudaEvent_t make() {
-    cudaEvent_t e = nullptr;
-    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    ev.push_back(e);
-    return e;
+    if (next == plan->n_events) {
+      cudaEvent_t e = nullptr;
+      if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      cudaEvent_t* grown = (cudaEvent_t*)realloc(plan->events, sizeof(cudaEvent_t) * (plan->n_events + 1));
+      if (!grown) {
+        cudaEventDestroy(e);
+        return nullptr;
+      }
+      plan->events = grown;
+      plan->events[plan->n_events++] = e;
+    }
+    return plan->events[next++];
   }
 };
 
@@ -77,10 +87,19 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
   if (first_group > group) first_group = group;
   const HostPassLayout L = make_layout(plan, group);
   if (workspace_bytes < L.total) return TRA_ERR_CAPACITY;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) return TRA_ERR_CUDA;
+  if (device != plan->device) return TRA_ERR_INVALID_ARG;     // the plan's tables and streams live on its device
   cudaStream_t cs = (cudaStream_t)stream_;
   if (!plan->copy_in) {   // the two copy streams live as long as the plan
-    TRA_CUDA_CHECK(cudaStreamCreateWithFlags(&plan->copy_in, cudaStreamNonBlocking));
-    TRA_CUDA_CHECK(cudaStreamCreateWithFlags(&plan->copy_out, cudaStreamNonBlocking));
+    cudaStream_t in = nullptr, out = nullptr;
+    TRA_CUDA_CHECK(cudaStreamCreateWithFlags(&in, cudaStreamNonBlocking));
+    if (cudaStreamCreateWithFlags(&out, cudaStreamNonBlocking) != cudaSuccess) {
+      cudaStreamDestroy(in);
+      return TRA_ERR_CUDA;
+    }
+    plan->copy_in = in;
+    plan->copy_out = out;
   }
   cudaStream_t s_in = plan->copy_in, s_out = plan->copy_out;
   uint8_t* ws = (uint8_t*)workspace;
@@ -88,7 +107,7 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
   const size_t head_bytes = S * d * 2;
   const int row_bytes = (int)(d * 2);
   const void* host_in[3] = {Q_host, K_host, V_host};
-  EventPool pool;
+  EventPool pool{plan};
 
   // the copy streams start after whatever the caller queued on its stream
   cudaEvent_t start = pool.make();

@@ -110,6 +110,8 @@ static void tra_plan_free(tra_plan* p) {
   cudaFree(p->d_status);
   if (p->copy_in) cudaStreamDestroy(p->copy_in);
   if (p->copy_out) cudaStreamDestroy(p->copy_out);
+  for (int i = 0; i < p->n_events; ++i) cudaEventDestroy(p->events[i]);
+  free(p->events);
   delete p;
 }
 
@@ -135,7 +137,9 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   p->N = T * H * W;
   p->S = p->N + cfg->n_text;
   p->NB = (p->S + cfg->block - 1) / cfg->block;
-  p->NBv = (p->N + cfg->block - 1) / cfg->block;
+  // video blocks: made of video tokens only when text follows (the block that holds both kinds is
+  // kept dense like a text block, so that every text key stays visible: Section 3.2, last paragraph)
+  p->NBv = cfg->n_text > 0 ? p->N / cfg->block : (p->N + cfg->block - 1) / cfg->block;
   p->z_tau = tra_inverse_normal_cdf(cfg->tau);
   if (cudaGetDevice(&p->device) != cudaSuccess) {
     delete p;
