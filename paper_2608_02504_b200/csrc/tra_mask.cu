@@ -392,7 +392,8 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 // ---------------------------------------------------------------------------------------
 #define TRA_PAIR_WINDOW 8
 #define TRA_PAIR_CHUNK 32
-#define TRA_PAIR_THREADS 256
+#define TRA_PAIR_THREADS 512
+#define TRA_PAIR_LOADS 24          // byte loads of one row a lane keeps in flight
 
 __global__ void __launch_bounds__(TRA_PAIR_THREADS)
 tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restrict__ pairs, int NB, int NT, int G,
@@ -402,32 +403,38 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
   const int win_rows = TRA_PAIR_CHUNK + TRA_PAIR_WINDOW;
   uint32_t* s_win = s_pair;                                                  // [win_rows][words]
   uint16_t* s_band = (uint16_t*)(s_win + win_rows * words);                  // [NT][window]
-  uint8_t* s_used = (uint8_t*)(s_band + (size_t)NT * TRA_PAIR_WINDOW);       // [NT]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long bh = blockIdx.x;
   const uint8_t* mask_h = block_mask + bh * NB * (long long)NB;
   int32_t* out = pairs + bh * ((NT + 1) / 2) * 2;
 
-  for (int t = tid; t < NT; t += TRA_PAIR_THREADS) s_used[t] = 0;
   for (int chunk0 = 0; chunk0 < NT; chunk0 += TRA_PAIR_CHUNK) {
     const int rows = min(win_rows, NT - chunk0);
     __syncthreads();                         // the previous chunk's window has been read
-    // one warp per window row; the loads of eight words of the row are in flight together
-    for (int r = warp; r < rows; r += TRA_PAIR_THREADS / 32) {
-      for (int wd0 = 0; wd0 < words; wd0 += 8) {
-        uint32_t on[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+    // one warp per window row; the loads of TRA_PAIR_LOADS words of the row are in flight together.
+    // The last rows of a window are the first rows of the next: they are moved, not read again.
+    const int keep = chunk0 > 0 ? TRA_PAIR_WINDOW : 0;
+    if (keep) {
+      for (int i = tid; i < keep * words; i += TRA_PAIR_THREADS) s_win[i] = s_win[TRA_PAIR_CHUNK * words + i];
+      __syncthreads();
+    }
+    for (int r = keep + warp; r < rows; r += TRA_PAIR_THREADS / 32) {
+      for (int wd0 = 0; wd0 < words; wd0 += TRA_PAIR_LOADS) {
+        uint32_t on[TRA_PAIR_LOADS];
+#pragma unroll
+        for (int q = 0; q < TRA_PAIR_LOADS; ++q) on[q] = 0u;
         for (int g = 0; g < G; ++g) {
           const int u = (chunk0 + r) * G + g;
           if (u >= NB) break;
           const uint8_t* row = mask_h + (long long)u * NB;
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {           // eight independent loads
+          for (int q = 0; q < TRA_PAIR_LOADS; ++q) {           // independent loads
             const int j = (wd0 + q) * 32 + lane;
             on[q] |= j < NB ? (uint32_t)row[j] : 0u;
           }
         }
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
+        for (int q = 0; q < TRA_PAIR_LOADS; ++q) {
           const uint32_t bits = __ballot_sync(0xffffffffu, on[q] != 0u);
           if (lane == 0 && wd0 + q < words) s_win[r * words + wd0 + q] = bits;
         }
@@ -451,35 +458,48 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
   }
   __syncthreads();
   if (warp != 0) return;
+  // Greedy matching by one warp.  The "matched" flags of all tiles live in registers: lane l holds the
+  // 64 tiles [64 l, 64 l + 64) (NT <= 2048), so a step costs a few shuffles and no shared-memory round trip.
+  unsigned long long used = 0ull;
+  auto first_free_from = [&](int from) -> int {          // the first unmatched tile >= from, or NT
+    unsigned long long free_bits = ~used;
+    const int lo = 64 * lane;
+    if (lo + 63 < from) free_bits = 0ull;
+    else if (lo < from) free_bits &= ~0ull << (from - lo);
+    if (lo >= NT) free_bits = 0ull;
+    else if (NT - lo < 64) free_bits &= (1ull << (NT - lo)) - 1ull;
+    const uint32_t cand = free_bits ? (uint32_t)(lo + __ffsll((long long)free_bits) - 1) : (uint32_t)NT;
+    return (int)__reduce_min_sync(0xffffffffu, cand);
+  };
+  auto mark = [&](int t) {
+    if (t >= 0 && lane == (t >> 6)) used |= 1ull << (t & 63);
+  };
   int n_out = 0;
-  for (int u = 0; u < NT; ++u) {
-    if (s_used[u]) continue;                 // the same for every lane
+  for (int u = first_free_from(0); u < NT; u = first_free_from(u + 1)) {
+    const int vc = min(u + 1 + lane, NT - 1);
+    const unsigned long long w = __shfl_sync(0xffffffffu, used, vc >> 6);
     uint32_t key = 0xffffffffu;              // (unshared blocks, window position) of this lane's candidate
-    if (lane < TRA_PAIR_WINDOW) {
-      const int v = u + 1 + lane;
-      if (v < NT && !s_used[v]) key = ((uint32_t)s_band[u * TRA_PAIR_WINDOW + lane] << 8) | (uint32_t)lane;
-    }
+    if (lane < TRA_PAIR_WINDOW && u + 1 + lane < NT && !((w >> (vc & 63)) & 1ull))
+      key = ((uint32_t)s_band[u * TRA_PAIR_WINDOW + lane] << 8) | (uint32_t)lane;
     key = __reduce_min_sync(0xffffffffu, key);
-    int v = -1;
+    int v;
     if (key != 0xffffffffu) {
       v = u + 1 + (int)(key & 0xffu);
     } else {                                 // nothing left in the window: the next unmatched tile, if any
-      for (int base = u + 1 + TRA_PAIR_WINDOW; base < NT && v < 0; base += 32) {
-        const int cand = base + lane;
-        const uint32_t free_mask = __ballot_sync(0xffffffffu, cand < NT && !s_used[cand]);
-        if (free_mask) v = base + __ffs(free_mask) - 1;
-      }
+      mark(u);
+      v = first_free_from(u + 1 + TRA_PAIR_WINDOW);
+      if (v >= NT) v = -1;
     }
+    mark(u);
+    mark(v);
     if (lane == 0 && TRA_IDX(n_out, (NT + 1) / 2, status) && (v == -1 || TRA_IDX(v, NT, status))) {
-      s_used[u] = 1;
-      if (v >= 0) s_used[v] = 1;
       out[2 * n_out] = u;
       out[2 * n_out + 1] = v;
     }
     ++n_out;
-    __syncwarp();
   }
 }
+
 
 extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* block_mask,
                                     int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
@@ -520,8 +540,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     const int G = (128 % b == 0) ? 128 / b : 1;
     const int NT = (NB + G - 1) / G;
     const size_t pair_smem = ((size_t)(TRA_PAIR_CHUNK + TRA_PAIR_WINDOW) * ((NB + 31) / 32)) * 4 +
-                             (size_t)NT * TRA_PAIR_WINDOW * 2 + (size_t)NT;
-    if (pair_smem > 200 * 1024) return TRA_ERR_UNSUPPORTED;
+                             (size_t)NT * TRA_PAIR_WINDOW * 2;
+    if (pair_smem > 200 * 1024 || NT > 2048) return TRA_ERR_UNSUPPORTED;
     if (pair_smem > 48 * 1024)
       TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)pair_smem));
