@@ -919,8 +919,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           const uint32_t all_runs = sa.x & sa.y & sa.z & sa.w & sb4.x & sb4.y & sb4.z & sb4.w;
           if (all_runs & (1u << 30)) {
             // A key (x0 + j, ys) is inside the disk iff |x0 + j - qx| <= w with
-            // w = floor(sqrt(theta - (ys - qy)^2)): one square root per slice, then an unsigned
-            // range test per key:  0 <= j + (x0 - qx + w) <= 2 w.
+            // w = floor(sqrt(theta - (ys - qy)^2)): one square root per slice gives the interval of
+            // inside keys, 0 <= j + (x0 - qx + w) <= 2 w, as a word of flags; one test per key.
 #pragma unroll
             for (int q = 0; q < BN / 16; ++q) {
               const uint32_t sw = slice_word(q);
@@ -930,11 +930,13 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               const int dy = tra_coord_y(sw) - qy;
               const int rem = th - dy * dy;
               const int w = tra_isqrt_small_nocvt(max(rem, 0));
-              const uint32_t base = rem < 0 ? 0x40000000u : (uint32_t)(w + tra_coord_x(sw) - qx);
-              const uint32_t span = (uint32_t)(2 * w);
+              // keys j with 0 <= j + bs <= 2 w are inside: one 16-bit word of "inside" flags per slice
+              const int bs = w + tra_coord_x(sw) - qx;
+              const int lo = max(-bs, 0), hi = min(2 * w - bs, 15);
+              const uint32_t inside = (rem >= 0 && hi >= lo) ? ((0xFFFFu >> (15 - hi)) & (0xFFFFu << lo)) : 0u;
 #pragma unroll
               for (int j = 0; j < 16; ++j)
-                if (base + (uint32_t)j > span) sb[q * 16 + j] = __float_as_uint(-1e30f);
+                if (((inside >> j) & 1u) == 0u) sb[q * 16 + j] = __float_as_uint(-1e30f);
             }
           } else if (one_frame) {       // every key of the block in one frame, some slice not a row run
 #pragma unroll
