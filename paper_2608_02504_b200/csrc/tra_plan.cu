@@ -47,7 +47,7 @@ __global__ void tra_count_table_kernel(int T, int H, int W, int n_radii,
   for (int delta = 0; delta < T; ++delta) c += tra_frame_count(y, x, H, W, th[delta]);
   size_t frame_stride = (size_t)H * W * n_radii;
   size_t base = (size_t)yx * n_radii + k;
-  const size_t n_counts = frame_stride * T;
+  [[maybe_unused]] const size_t n_counts = frame_stride * T;
   if (TRA_IDX(base, n_counts, status)) counts[base] = c;  // f = 0
   for (int f = 0; f + 1 < T; ++f) {
     c += tra_frame_count(y, x, H, W, th[f + 1]);
