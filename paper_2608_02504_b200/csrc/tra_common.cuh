@@ -15,7 +15,7 @@ struct tra_box_t {
 };
 static_assert(sizeof(tra_box_t) == 16, "box is one 16-byte load");
 
-struct tra_block_boxes_t {
+struct __align__(16) tra_block_boxes_t {
   tra_box_t box[TRA_MAX_SEG];
   int32_t n_box;
   int32_t pad[3];
@@ -43,6 +43,11 @@ struct tra_plan {
   uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)
   uint32_t* d_counts_coarse;      // [T*H*W][16] every eighth entry of a row (n_radii <= 128), else NULL
   tra_block_boxes_t* d_boxes;     // [NB]
+  uint16_t* d_field_pos;          // where the block vote writes the count of frame cell (y, x), as an index into
+                                  // the frame's positions in tile-major order (the order repeats frame by frame):
+                                  // field_quads = 1: [H][W/4] index / 4 of the cells (y, 4j .. 4j+3), which are four
+                                  // consecutive positions starting at a multiple of four; else [H][W] one per cell
+  int field_quads;
   int* d_status;                  // device status word
   // copy streams and events of tra_hot_path_host, created on its first calls with this plan and kept
   cudaStream_t copy_in, copy_out;
@@ -56,6 +61,11 @@ __host__ __device__ inline uint32_t tra_pack_coord(int t, int y, int x) {
 __host__ __device__ inline int tra_coord_x(uint32_t c) { return (int)(c & 1023u); }
 __host__ __device__ inline int tra_coord_y(uint32_t c) { return (int)((c >> 10) & 1023u); }
 __host__ __device__ inline int tra_coord_t(uint32_t c) { return (int)(c >> 20); }
+
+// Words per row of the block vote's count field: at least W + 1 (its difference array writes column
+// W), a whole number of 16-byte vectors, and an odd number of them so that threads that walk
+// neighbouring rows with 16-byte accesses fall into different shared-memory banks.
+__host__ __device__ inline int tra_field_row_words(int W) { return 4 * (((W + 4) / 4) | 1); }
 
 #define TRA_CUDA_CHECK(expr)                      \
   do {                                            \

@@ -25,10 +25,12 @@
 //    c(y', x') = #{queries i : (x'-x_i)^2 + (y'-y_i)^2 <= theta[ridx_i][|f - t_i|]} is built for
 //    the whole frame at once: a query's disk meets row y' in the x-interval of half-width
 //    floor(sqrt(theta - (y'-y_i)^2)), which adds +1 / -1 to a difference array in shared
-//    memory; a prefix sum along each row turns it into the counts (a disk that covers the whole
-//    frame is only counted once, a disk that covers a whole row skips the square root).  Every undecided key block
-//    then reads the counts of its own keys in that frame (c_j by definition) and accumulates
-//    its numbers of reached and of high columns.  When the query block lies in one frame t0 the
+//    memory (rows y_i - dy and y_i + dy share the half-width; a disk that covers the whole frame
+//    is only counted once).  One thread per row then takes the running sum along the row and
+//    stores the counts as bytes in the frame's tile-major order, so that the keys of a block are
+//    consecutive bytes.  Every undecided key block then reads the counts of its own keys in that
+//    frame (c_j by definition), four per 32-bit word, and compares all four with the two
+//    thresholds at once (adding 127 - t to a byte sets its top bit iff the byte exceeds t).  When the query block lies in one frame t0 the
 //    frames t0 - k and t0 + k see the same thresholds, so one field serves both.
 // The outcome equals the unpruned vote bit for bit.
 // ---------------------------------------------------------------------------------------
@@ -40,29 +42,36 @@ __device__ __forceinline__ int tra_isqrt_small(int n) {
   return (int)r;
 }
 
+// kQuads: the plan's position table has one entry per four cells of a row (see tra_plan::d_field_pos).
+template <bool kQuads>
 __global__ void __launch_bounds__(TRA_MASK_THREADS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
-                      uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int S, int NB,
+                      const uint16_t* __restrict__ field_pos, uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int S, int NB,
                       int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal,
                       int* __restrict__ status) {
   extern __shared__ int32_t s_dyn[];
-  __shared__ int s_rank_ridx[128];
+  __shared__ __align__(16) int s_rank_key[128];
   __shared__ uint32_t s_sorted[128];        // queries in descending candidate index: coord | 0, and ...
   __shared__ uint16_t s_sorted_r[128];      // ... their candidate index
   __shared__ tra_block_boxes_t s_ubox;
-  __shared__ int s_rstar, s_count, s_whole;
+  __shared__ int s_rstar, s_count, s_whole[2];
 
-  const int Wp = (W + 1) | 1;                                      // odd row stride
+  const int Wp = tra_field_row_words(W);
   const int Tp = (T + 3) & ~3;                                     // keeps s_diff 16-byte aligned
-  const int n_diff = (H * Wp + 3) & ~3;                            // words of the count field, padded to 16 bytes
+  const int n_diff = H * Wp;                                       // words of the count field
   int32_t* s_theta_star = s_dyn;                                   // [T]
   int32_t* s_frame_ylo = s_dyn + Tp;                               // [T] rows of the frame that hold keys of an
   int32_t* s_frame_yhi = s_dyn + 2 * Tp;                           // [T] undecided key block (yhi < 0: none)
-  int32_t* s_diff = s_dyn + 3 * Tp;                                // [H * (W + 1)]
+  int32_t* s_diff = s_dyn + 3 * Tp;                                // [H][Wp]
   uint16_t* s_ne = (uint16_t*)(s_diff + n_diff);                   // [NB] reached columns
   uint16_t* s_hi = s_ne + NB;                                      // [NB] high columns
   uint8_t* s_state = (uint8_t*)(s_hi + NB);                        // [NB] 0 / 1 decided, 2 undecided
+  const int HW = H * W;
+  const int n_pos = kQuads ? HW / 4 : HW;                          // entries of the position table
+  uint32_t* s_cnt = (uint32_t*)(s_dyn + 3 * Tp + n_diff + (5 * NB + 15) / 16 * 4);   // [H * W] bytes (16-byte
+                                                                   // aligned): counts in tile-major order
+  uint16_t* s_pos = (uint16_t*)(s_cnt + (HW + 15) / 16 * 4);       // [n_pos] the plan's position table
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x;
@@ -79,7 +88,6 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   const int q0 = u * b;
   const int nq = min(b, N - q0);                       // valid queries of this block
   const int need = b / 3 + 1;
-  const int HW = H * W;
 
   // this thread's query
   int qx = 0, qy = 0, qt = 0, qr = 0;
@@ -89,8 +97,11 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     qy = tra_coord_y(c);
     qt = tra_coord_t(c);
     qr = min((int)ridx_h[q0 + tid], n_radii - 1);      // a candidate index past the table reads its last row
-    s_rank_ridx[tid] = qr;
   }
+  // sort key: candidate index, then lane order (unique per query); -1 for the threads without a query
+  s_rank_key[tid] = tid < nq ? (qr << 7) | (TRA_MASK_THREADS - 1 - tid) : -1;
+  for (int i = tid; i < (n_pos + 7) / 8; i += TRA_MASK_THREADS)
+    reinterpret_cast<uint4*>(s_pos)[i] = __ldg(reinterpret_cast<const uint4*>(field_pos) + i);
 #ifdef TRA_DEBUG
   if (tid < nq && (qx >= W || qy >= H || qt >= T)) tra_set_status(status, TRA_ERR_BOUNDS);   // indexes the count field
 #endif
@@ -113,10 +124,12 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   // the queries to the threads in descending candidate order, so that the threads of a warp draw
   // disks of similar size (the row loops below run as long as the largest disk of the warp).
   if (tid < nq) {
+    const int key = (qr << 7) | (TRA_MASK_THREADS - 1 - tid);
     int rank = 0;
-    for (int j = 0; j < nq; ++j) {
-      int o = s_rank_ridx[j];
-      rank += (o > qr) || (o == qr && j < tid);
+#pragma unroll 4
+    for (int j = 0; j < TRA_MASK_THREADS / 4; ++j) {
+      const int4 o = reinterpret_cast<const int4*>(s_rank_key)[j];
+      rank += (o.x > key) + (o.y > key) + (o.z > key) + (o.w > key);
     }
     if (rank == need - 1) s_rstar = qr;
     if (TRA_IDX(rank, nq, status)) {
@@ -141,10 +154,12 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   int kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
     int decided = 0;   // 0 = vote 0, 1 = vote 1, 2 = undecided
+    tra_block_boxes_t vb;
+    vb.n_box = 0;
     if (v >= NBv) {
       decided = 1;     // text key block
     } else if (rstar >= 0) {
-      tra_block_boxes_t vb = boxes[v];
+      vb = boxes[v];
       bool all_reject = true, all_accept = true;
       for (int iu = 0; iu < s_ubox.n_box; ++iu) {
         const tra_box_t a = s_ubox.box[iu];
@@ -167,7 +182,6 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     s_state[v] = (uint8_t)decided;
     if (decided == 2) {
       // frames this key block has tokens in, and the rows of each that hold them
-      const tra_block_boxes_t vb = boxes[v];
       for (int iv = 0; iv < vb.n_box; ++iv)
         for (int f = vb.box[iv].t0; f <= vb.box[iv].t1; ++f) {
           if (!TRA_IDX(f, T, status)) break;
@@ -183,92 +197,94 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   __syncthreads();
 
   // ---- 2. count field of every frame that holds an undecided key block ---------------------
-  // builds the field for the frame distance dist(thread) -> |f - t_i| of every query
+  // builds the field for the frame distance dist(thread) -> |f - t_i| of every query and returns the
+  // number of queries whose disk covers the whole frame (they are left out of the field).
   // Only the rows win_lo .. win_hi of the frame are read afterwards: the field is built for them alone.
+  int n_field = 0;
   auto build_field = [&](auto dist_of_query, int win_lo, int win_hi) {
-    for (int i = (win_lo * Wp) / 4 + tid; i < ((win_hi + 1) * Wp + 3) / 4; i += TRA_MASK_THREADS)
+    const int th = tid < nq ? __ldg(theta + qr * T + dist_of_query()) : 0;   // in flight during the zeroing
+    int* whole = &s_whole[n_field++ & 1];   // alternates: the last field's readers may still be counting
+    const int row4 = Wp / 4;
+    for (int i = win_lo * row4 + tid; i < (win_hi + 1) * row4; i += TRA_MASK_THREADS)
       reinterpret_cast<uint4*>(s_diff)[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (tid == 0) s_whole = 0;
+    if (tid == 0) *whole = 0;
     __syncthreads();
     if (tid < nq) {
-      const int th = __ldg(theta + qr * T + dist_of_query());
       const int far_x = max(qx, W - 1 - qx), far_y = max(qy, H - 1 - qy);
       if (th >= far_x * far_x + far_y * far_y) {
-        atomicAdd(&s_whole, 1);                       // the disk covers the whole frame
+        atomicAdd(whole, 1);                          // the disk covers the whole frame
       } else {
+        // rows qy - dy and qy + dy meet the disk in the same x-interval: one half-width serves both
+        // (a half-width that reaches both frame edges clamps to the whole row by itself)
         const int R = tra_isqrt_small(th);
-        const int ylo = max(win_lo, qy - R), yhi = min(win_hi, qy + R);
-        for (int yy = ylo; yy <= yhi; ++yy) {
-          const int dy = yy - qy;
-          const int rem = th - dy * dy;
-          int lo = 0, hi = W;                         // the disk covers the whole row ...
-          if (rem < far_x * far_x) {                  // ... unless its half-width falls short
-            const int w = tra_isqrt_small(rem);
-            lo = max(0, qx - w);
-            hi = min(W - 1, qx + w) + 1;
+        const int d_first = max(0, max(win_lo - qy, qy - win_hi));
+        const int d_last = min(R, max(qy - win_lo, win_hi - qy));
+        const unsigned span = (unsigned)(win_hi - win_lo);
+        for (int dy = d_first; dy <= d_last; ++dy) {
+          const int w = tra_isqrt_small(th - dy * dy);
+          const int lo = max(0, qx - w), hi = min(W - 1, qx + w) + 1;      // lo < hi <= W < Wp
+          const int ya = qy - dy, yb = qy + dy;
+          if ((unsigned)(ya - win_lo) <= span && TRA_IDX(ya * Wp + hi, H * Wp, status)) {
+            atomicAdd(&s_diff[ya * Wp + lo], 1);
+            atomicAdd(&s_diff[ya * Wp + hi], -1);
           }
-          if (!TRA_IDX(yy * Wp + hi, H * Wp, status)) continue;      // lo <= hi <= W < Wp
-          atomicAdd(&s_diff[yy * Wp + lo], 1);
-          atomicAdd(&s_diff[yy * Wp + hi], -1);
+          if (dy > 0 && (unsigned)(yb - win_lo) <= span && TRA_IDX(yb * Wp + hi, H * Wp, status)) {
+            atomicAdd(&s_diff[yb * Wp + lo], 1);
+            atomicAdd(&s_diff[yb * Wp + hi], -1);
+          }
         }
       }
     }
     __syncthreads();
-    // prefix sum along x: two threads (a lane pair) per row, each over half of it; the second adds
-    // the first one's total (the row stride W + 1 is odd, so the threads of a warp walk different banks)
-    {
-      const int half_w = (W + 1) >> 1;
-      for (int yy0 = win_lo; yy0 <= win_hi; yy0 += TRA_MASK_THREADS / 2) {
-        const int yy = yy0 + (tid >> 1), part = tid & 1;
-        const bool on = yy <= win_hi;
-        int32_t* row = s_diff + (on ? yy : 0) * Wp;
-        const int xa = part ? half_w : 0, xb = part ? W : half_w;
-        int run = 0;
-        for (int x0 = xa; x0 < xb && on; x0 += 8) {   // eight independent loads, then the running sum
-          int v[8];
-#pragma unroll
-          for (int j = 0; j < 8; ++j) v[j] = x0 + j < xb ? row[x0 + j] : 0;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) {
-            run += v[j];
-            if (x0 + j < xb) row[x0 + j] = run;
-          }
+    // running sum along x, one thread per row; the counts (at most b <= 128) go out as bytes in tile-major order
+    for (int yy = win_lo + tid; yy <= win_hi; yy += TRA_MASK_THREADS) {
+      uint32_t run = 0;
+      if constexpr (kQuads) {
+        const uint4* row = reinterpret_cast<const uint4*>(s_diff + yy * Wp);
+        const uint16_t* pos = s_pos + yy * (W / 4);
+#pragma unroll 4
+        for (int j = 0; j < W / 4; ++j) {
+          const uint4 v = row[j];
+          const uint32_t c0 = run + v.x, c1 = c0 + v.y, c2 = c1 + v.z, c3 = c2 + v.w;
+          run = c3;
+          if (TRA_IDX(pos[j], HW / 4, status)) s_cnt[pos[j]] = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
         }
-        const int left = __shfl_xor_sync(0xffffffffu, run, 1);       // the other half's total
-        if (on && part)
-          for (int x = xa; x < xb; ++x) row[x] += left;
+      } else {
+        const int32_t* row = s_diff + yy * Wp;
+        const uint16_t* pos = s_pos + yy * W;
+        for (int x = 0; x < W; ++x) {
+          run += (uint32_t)row[x];
+          if (TRA_IDX(pos[x], HW, status)) reinterpret_cast<uint8_t*>(s_cnt)[pos[x]] = (uint8_t)run;
+        }
       }
     }
     __syncthreads();
+    return *whole;
   };
-  // undecided key blocks with tokens in frame f read the field: one warp per block
-  auto count_frame = [&](int f) {
-    const int whole = s_whole;                         // queries whose disk covers every key of the frame
+  // undecided key blocks with tokens in frame f read their keys' counts: one warp per block, four keys
+  // per lane and word.  A count c (without the `whole` queries) is reached iff c > -whole and high iff
+  // c > floor(b/3) - whole; with t >= -1 the byte c + (127 - t) <= 255 has its top bit set iff c > t
+  // (c <= b - whole, and t = -1 only when whole >= 1).
+  auto count_frame = [&](int f, int whole) {
+    const uint32_t add_reached = 0x01010101u * (uint32_t)(127 - max(-whole, -1));
+    const uint32_t add_high = 0x01010101u * (uint32_t)(127 - max(b / 3 - whole, -1));
     const int p_begin = f * HW, p_end = min(N, (f + 1) * HW);
     const int v_first = p_begin / b, v_last = (p_end - 1) / b;     // video blocks only: p_end <= N
     for (int v = v_first + warp; v <= v_last; v += TRA_MASK_WARPS) {
       if (s_state[v] != 2) continue;
-      const int ps = max(v * b, p_begin), pe = min((v + 1) * b, p_end);
-      int ne = 0, hi = 0;
-      // b <= 128: at most four keys per lane; their coordinate loads are in flight together
-      uint32_t kc[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int p = ps + 32 * i + lane;
-        kc[i] = p < pe ? __ldg(coord_packed + p) : 0xffffffffu;
+      const int i0 = max(v * b, p_begin) - p_begin, i1 = min((v + 1) * b, p_end) - p_begin;   // bytes [i0, i1)
+      int acc = 0;                                        // reached | high << 16 of this lane's keys
+      for (int wd = (i0 >> 2) + lane; 4 * wd < i1; wd += 32) {
+        const uint32_t x = s_cnt[wd];
+        uint32_t m = 0x80808080u;                         // bytes of the word that belong to [i0, i1)
+        if (i0 > 4 * wd) m &= 0xffffffffu << (8 * (i0 - 4 * wd));
+        if (i1 < 4 * wd + 4) m &= 0xffffffffu >> (8 * (4 * wd + 4 - i1));
+        acc += __popc((x + add_reached) & m) + (__popc((x + add_high) & m) << 16);
       }
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        if (ps + 32 * i >= pe) break;                     // uniform across the warp
-        int c = 0;
-        if (kc[i] != 0xffffffffu && TRA_IDX(tra_coord_y(kc[i]) * Wp + tra_coord_x(kc[i]), H * Wp, status))
-          c = s_diff[tra_coord_y(kc[i]) * Wp + tra_coord_x(kc[i])] + whole;
-        ne += __popc(__ballot_sync(0xffffffffu, c > 0));
-        hi += __popc(__ballot_sync(0xffffffffu, 3 * c > b));
-      }
+      acc = __reduce_add_sync(0xffffffffu, acc);
       if (lane == 0) {            // one warp owns v inside a frame; frames are processed in turn
-        s_ne[v] = (uint16_t)(s_ne[v] + ne);
-        s_hi[v] = (uint16_t)(s_hi[v] + hi);
+        s_ne[v] = (uint16_t)(s_ne[v] + (acc & 0xffff));
+        s_hi[v] = (uint16_t)(s_hi[v] + (acc >> 16));
       }
     }
   };
@@ -287,21 +303,20 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       int win_lo = min(need_a ? s_frame_ylo[fa] : H, need_b ? s_frame_ylo[fb] : H);
       int win_hi = max(need_a ? s_frame_yhi[fa] : -1, need_b ? s_frame_yhi[fb] : -1);
       if (!TRA_IDX(win_lo, H, status) || !TRA_IDX(win_hi, H, status)) win_lo = 0, win_hi = H - 1;
-      build_field([&]() { return k; }, win_lo, win_hi);
-      if (need_a) count_frame(fa);
-      if (need_b) count_frame(fb);
-      __syncthreads();
+      const int whole = build_field([&]() { return k; }, win_lo, win_hi);
+      if (need_a) count_frame(fa, whole);
+      if (need_b) count_frame(fb, whole);
     }
   } else {
     for (int f = 0; f < T; ++f) {
       if (s_frame_yhi[f] < 0) continue;                 // uniform across the CTA
-      build_field([&]() { return abs(qt - f); }, s_frame_ylo[f], s_frame_yhi[f]);
-      count_frame(f);
-      __syncthreads();
+      const int whole = build_field([&]() { return abs(qt - f); }, s_frame_ylo[f], s_frame_yhi[f]);
+      count_frame(f, whole);
     }
   }
 
   // ---- 3. votes of the undecided key blocks -------------------------------------------------
+  __syncthreads();
   kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
     if (s_state[v] != 2) continue;
@@ -514,17 +529,17 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   const long long rows = BH * NB;
 
   const int H = plan->cfg.H, W = plan->cfg.W;
-  size_t smem = ((size_t)3 * ((T + 3) & ~3) + (((size_t)H * ((W + 1) | 1) + 3) & ~(size_t)3)) * sizeof(int32_t) +
-                (size_t)NB * 5;
-  smem = (smem + 15) & ~(size_t)15;
-  if (smem > 200 * 1024) return TRA_ERR_UNSUPPORTED;     // frame too large for the count field
+  size_t smem = ((size_t)3 * ((T + 3) & ~3) + (size_t)H * tra_field_row_words(W)) * sizeof(int32_t) +
+                ((size_t)NB * 5 + 15) / 16 * 16 + ((size_t)H * W + 15) / 16 * 16 +
+                ((((size_t)H * W / (plan->field_quads ? 4 : 1)) + 7) & ~(size_t)7) * sizeof(uint16_t);
+  if (smem > 200 * 1024 || !plan->d_field_pos) return TRA_ERR_UNSUPPORTED;   // frame too large for the count field
   dim3 grid((unsigned)NB, (unsigned)BH);
+  auto vote = plan->field_quads ? tra_block_vote_kernel<true> : tra_block_vote_kernel<false>;
   if (smem > 48 * 1024)
-    TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_block_vote_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)smem));
-  tra_block_vote_kernel<<<grid, TRA_MASK_THREADS, smem, stream>>>(
-      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, block_mask, row_ptr, plan->N, plan->S, NB,
-      plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0,
+    TRA_CUDA_CHECK(cudaFuncSetAttribute(vote, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  vote<<<grid, TRA_MASK_THREADS, smem, stream>>>(
+      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, plan->d_field_pos, block_mask, row_ptr, plan->N, plan->S,
+      NB, plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0,
       plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,

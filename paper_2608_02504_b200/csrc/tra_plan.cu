@@ -107,6 +107,7 @@ static void tra_plan_free(tra_plan* p) {
   cudaFree(p->d_counts);
   cudaFree(p->d_counts_coarse);
   cudaFree(p->d_boxes);
+  cudaFree(p->d_field_pos);
   cudaFree(p->d_status);
   if (p->copy_in) cudaStreamDestroy(p->copy_in);
   if (p->copy_out) cudaStreamDestroy(p->copy_out);
@@ -269,6 +270,22 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
     if (run) slices[si] = tra_pack_coord(t, y, x) | (1u << 30);
   }
 
+  // block vote: where the count of a frame cell goes in the frame's tile-major order
+  std::vector<uint16_t> field_pos;
+  const bool field_pos_fits = (long long)H * W <= 65535;
+  if (field_pos_fits) {
+    std::vector<int32_t> pos_of((size_t)H * W);
+    for (int i = 0; i < H * W; ++i) pos_of[(size_t)p->h_coord[3 * i + 1] * W + p->h_coord[3 * i + 2]] = i;
+    bool quads = W % 4 == 0;
+    for (int c = 0; c < H * W && quads; c += 4)
+      quads = pos_of[c] % 4 == 0 && pos_of[c + 1] == pos_of[c] + 1 && pos_of[c + 2] == pos_of[c] + 2 &&
+              pos_of[c + 3] == pos_of[c] + 3;
+    p->field_quads = quads ? 1 : 0;
+    const size_t n = quads ? (size_t)H * W / 4 : (size_t)H * W;
+    field_pos.assign((n + 7) & ~(size_t)7, 0);
+    for (size_t i = 0; i < n; ++i) field_pos[i] = (uint16_t)(quads ? pos_of[4 * i] / 4 : pos_of[i]);
+  }
+
   // device tables
   const size_t count_elems = (size_t)p->N * nr;
   bool ok = cudaMalloc(&p->d_coord_packed, sizeof(uint32_t) * (p->N + 128)) == cudaSuccess &&
@@ -279,6 +296,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
             cudaMalloc(&p->d_counts, sizeof(uint32_t) * count_elems) == cudaSuccess &&
             (nr > 128 || cudaMalloc(&p->d_counts_coarse, sizeof(uint32_t) * 16 * (size_t)p->N) == cudaSuccess) &&
             cudaMalloc(&p->d_boxes, sizeof(tra_block_boxes_t) * p->NB) == cudaSuccess &&
+            (!field_pos_fits || cudaMalloc(&p->d_field_pos, sizeof(uint16_t) * field_pos.size()) == cudaSuccess) &&
             cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess;
   ok = ok &&
        cudaMemcpyAsync(p->d_coord_packed, packed.data(), sizeof(uint32_t) * (p->N + 128),
@@ -293,6 +311,8 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&
        cudaMemcpyAsync(p->d_boxes, boxes.data(), sizeof(tra_block_boxes_t) * p->NB,
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+       (!field_pos_fits || cudaMemcpyAsync(p->d_field_pos, field_pos.data(), sizeof(uint16_t) * field_pos.size(),
+                                           cudaMemcpyHostToDevice, stream) == cudaSuccess) &&
        cudaMemsetAsync(p->d_status, 0, sizeof(int), stream) == cudaSuccess;
   if (ok) {
     int total = H * W * nr;
