@@ -64,9 +64,8 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   int32_t* s_frame_ylo = s_dyn + Tp;                               // [T] rows of the frame that hold keys of an
   int32_t* s_frame_yhi = s_dyn + 2 * Tp;                           // [T] undecided key block (yhi < 0: none)
   int32_t* s_diff = s_dyn + 3 * Tp;                                // [H][Wp]
-  uint16_t* s_ne = (uint16_t*)(s_diff + n_diff);                   // [NB] reached columns
-  uint16_t* s_hi = s_ne + NB;                                      // [NB] high columns
-  uint8_t* s_state = (uint8_t*)(s_hi + NB);                        // [NB] 0 / 1 decided, 2 undecided
+  uint32_t* s_cols = (uint32_t*)(s_diff + n_diff);                 // [NB] reached columns | high columns << 16
+  uint8_t* s_state = (uint8_t*)(s_cols + NB);                      // [NB] 0 / 1 decided, 2 undecided
   const int HW = H * W;
   const int n_pos = kQuads ? HW / 4 : HW;                          // entries of the position table
   uint32_t* s_cnt = (uint32_t*)(s_dyn + 3 * Tp + n_diff + (5 * NB + 15) / 16 * 4);   // [H * W] bytes (16-byte
@@ -115,8 +114,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     s_frame_yhi[i] = -1;
   }
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
-    s_ne[v] = 0;
-    s_hi[v] = 0;
+    s_cols[v] = 0;
   }
   __syncthreads();
 
@@ -274,18 +272,20 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       if (s_state[v] != 2) continue;
       const int i0 = max(v * b, p_begin) - p_begin, i1 = min((v + 1) * b, p_end) - p_begin;   // bytes [i0, i1)
       int acc = 0;                                        // reached | high << 16 of this lane's keys
-      for (int wd = (i0 >> 2) + lane; 4 * wd < i1; wd += 32) {
-        const uint32_t x = s_cnt[wd];
-        uint32_t m = 0x80808080u;                         // bytes of the word that belong to [i0, i1)
-        if (i0 > 4 * wd) m &= 0xffffffffu << (8 * (i0 - 4 * wd));
-        if (i1 < 4 * wd + 4) m &= 0xffffffffu >> (8 * (4 * wd + 4 - i1));
-        acc += __popc((x + add_reached) & m) + (__popc((x + add_high) & m) << 16);
+      if (((i0 | i1) & 3) == 0 && i1 - i0 == 128) {       // 32 whole words, one per lane (uniform across the warp)
+        const uint32_t x = s_cnt[(i0 >> 2) + lane];
+        acc = __popc((x + add_reached) & 0x80808080u) + (__popc((x + add_high) & 0x80808080u) << 16);
+      } else {
+        for (int wd = (i0 >> 2) + lane; 4 * wd < i1; wd += 32) {
+          const uint32_t x = s_cnt[wd];
+          uint32_t m = 0x80808080u;                       // bytes of the word that belong to [i0, i1)
+          if (i0 > 4 * wd) m &= 0xffffffffu << (8 * (i0 - 4 * wd));
+          if (i1 < 4 * wd + 4) m &= 0xffffffffu >> (8 * (4 * wd + 4 - i1));
+          acc += __popc((x + add_reached) & m) + (__popc((x + add_high) & m) << 16);
+        }
       }
       acc = __reduce_add_sync(0xffffffffu, acc);
-      if (lane == 0) {            // one warp owns v inside a frame; frames are processed in turn
-        s_ne[v] = (uint16_t)(s_ne[v] + (acc & 0xffff));
-        s_hi[v] = (uint16_t)(s_hi[v] + (acc >> 16));
-      }
+      if (lane == 0) s_cols[v] += (uint32_t)acc;   // one warp owns v inside a frame; frames are processed in turn
     }
   };
   // A query block that lies in one frame t0 sees frames t0 - k and t0 + k at the same distance:
@@ -320,7 +320,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
     if (s_state[v] != 2) continue;
-    const int ne = s_ne[v], hi = s_hi[v];
+    const int ne = (int)(s_cols[v] & 0xffffu), hi = (int)(s_cols[v] >> 16);
     const int keep = (ne > 0) && (10 * hi > 6 * ne);
     mask_row[v] = (uint8_t)keep;
     kept += keep;
