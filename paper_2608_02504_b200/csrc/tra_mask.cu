@@ -108,7 +108,10 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     s_ubox = boxes[u];
     s_count = 0;
     s_rstar = -1;
+    s_whole[0] = s_whole[1] = 0;
   }
+  for (int i = tid; i < n_diff / 4; i += TRA_MASK_THREADS)   // the prefix pass leaves the rows it read zeroed again
+    reinterpret_cast<uint4*>(s_diff)[i] = make_uint4(0u, 0u, 0u, 0u);
   for (int i = tid; i < T; i += TRA_MASK_THREADS) {
     s_frame_ylo[i] = H;
     s_frame_yhi[i] = -1;
@@ -200,13 +203,11 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   // Only the rows win_lo .. win_hi of the frame are read afterwards: the field is built for them alone.
   int n_field = 0;
   auto build_field = [&](auto dist_of_query, int win_lo, int win_hi) {
-    const int th = tid < nq ? __ldg(theta + qr * T + dist_of_query()) : 0;   // in flight during the zeroing
-    int* whole = &s_whole[n_field++ & 1];   // alternates: the last field's readers may still be counting
-    const int row4 = Wp / 4;
-    for (int i = win_lo * row4 + tid; i < (win_hi + 1) * row4; i += TRA_MASK_THREADS)
-      reinterpret_cast<uint4*>(s_diff)[i] = make_uint4(0u, 0u, 0u, 0u);
-    if (tid == 0) *whole = 0;
-    __syncthreads();
+    // The field is all zero here (set at the start, and again by every prefix pass), and no warp still
+    // reads it: warps that lag behind are counting, which reads the byte array only.
+    const int th = tid < nq ? __ldg(theta + qr * T + dist_of_query()) : 0;
+    int* whole = &s_whole[n_field & 1];     // alternates: the last field's readers may still be counting
+    int* whole_next = &s_whole[++n_field & 1];
     if (tid < nq) {
       const int far_x = max(qx, W - 1 - qx), far_y = max(qy, H - 1 - qy);
       if (th >= far_x * far_x + far_y * far_y) {
@@ -234,26 +235,32 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       }
     }
     __syncthreads();
-    // running sum along x, one thread per row; the counts (at most b <= 128) go out as bytes in tile-major order
+    if (tid == 0) *whole_next = 0;          // its last readers passed the barrier above
+    // running sum along x, one thread per row; the counts (at most b <= 128) go out as bytes in tile-major
+    // order, and the row (column W included) is zeroed for the next field
     for (int yy = win_lo + tid; yy <= win_hi; yy += TRA_MASK_THREADS) {
       uint32_t run = 0;
       if constexpr (kQuads) {
-        const uint4* row = reinterpret_cast<const uint4*>(s_diff + yy * Wp);
+        uint4* row = reinterpret_cast<uint4*>(s_diff + yy * Wp);
         const uint16_t* pos = s_pos + yy * (W / 4);
 #pragma unroll 4
         for (int j = 0; j < W / 4; ++j) {
           const uint4 v = row[j];
+          row[j] = make_uint4(0u, 0u, 0u, 0u);
           const uint32_t c0 = run + v.x, c1 = c0 + v.y, c2 = c1 + v.z, c3 = c2 + v.w;
           run = c3;
           if (TRA_IDX(pos[j], HW / 4, status)) s_cnt[pos[j]] = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
         }
+        row[W / 4] = make_uint4(0u, 0u, 0u, 0u);
       } else {
-        const int32_t* row = s_diff + yy * Wp;
+        int32_t* row = s_diff + yy * Wp;
         const uint16_t* pos = s_pos + yy * W;
         for (int x = 0; x < W; ++x) {
           run += (uint32_t)row[x];
+          row[x] = 0;
           if (TRA_IDX(pos[x], HW, status)) reinterpret_cast<uint8_t*>(s_cnt)[pos[x]] = (uint8_t)run;
         }
+        row[W] = 0;
       }
     }
     __syncthreads();
