@@ -607,7 +607,8 @@ def run_workload(api, name, dev, peak_tf, reps=2, gamma=None):
            "block_density": round(pairs_sparse / pairs_dense, 4),
            "speedup_sparse_vs_dense_plain": round(t["dense_plain"] / t["sparse"], 3),
            "mask_radius_overhead_frac_one_layer": round(
-               (t["budget_radius"] + t["block_mask"]) / (t["sparse"] + t["budget_radius"] + t["block_mask"]), 4)}
+               (t["budget_radius"] + t["block_mask"]) / (t["sparse"] + t["budget_radius"] + t["block_mask"]), 4),
+           "cta_key_block_lists": pairing_stats(bufs[0], bufs[4], block)}
     plan.close()
     return out
 

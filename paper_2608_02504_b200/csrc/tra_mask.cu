@@ -404,78 +404,83 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 // retains leaves the other tile idle.  This kernel pairs tiles with similar lists: one CTA per
 // (batch, head); tile t covers the query blocks [t G, (t + 1) G), G = 128 / block.
 //   1. row bitmaps of a window of tiles are built in shared memory (ballots over the byte mask),
-//      and for every tile u the number of key blocks that u and u + 1 + c do not share is
-//      stored for c = 0 .. kPairWindow - 1;
+//      and for every tile u the number of key blocks that u and each of its candidates do not
+//      share is stored.  The candidates are the next TRA_PAIR_WINDOW tiles and, when a frame holds
+//      more tiles than that, the three tiles about one frame ahead (the same place in the next
+//      frame: with a slow temporal decay those share far more key blocks than spatial neighbours);
 //   2. one warp matches the tiles greedily in ascending order: the first unmatched tile takes the
-//      unmatched tile of its window with the fewest unshared key blocks, or, when the window has
-//      none left, the next unmatched tile after it.  Every tile is matched (one is left alone
+//      unmatched candidate with the fewest unshared key blocks, or, when none is left, the next
+//      unmatched tile after the window.  Every tile is matched (one is left alone
 //      when their number is odd): pairs[i] = (u, v) for i < ceil(NT / 2), v = -1 for a lone tile.
 // Any perfect matching gives the same attention output; the choice only moves time.
 // ---------------------------------------------------------------------------------------
 #define TRA_PAIR_WINDOW 8
+#define TRA_PAIR_CANDS (TRA_PAIR_WINDOW + 3)
 #define TRA_PAIR_CHUNK 32
 #define TRA_PAIR_THREADS 512
 #define TRA_PAIR_LOADS 24          // byte loads of one row a lane keeps in flight
 
 __global__ void __launch_bounds__(TRA_PAIR_THREADS)
 tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restrict__ pairs, int NB, int NT, int G,
-                      int* __restrict__ status) {
+                      int frame_tiles, int* __restrict__ status) {
   extern __shared__ uint32_t s_pair[];
   const int words = (NB + 31) >> 5;
-  const int win_rows = TRA_PAIR_CHUNK + TRA_PAIR_WINDOW;
+  // candidate c of tile u is u + 1 + c for c < TRA_PAIR_WINDOW, then u + frame_tiles - 1, + 0, + 1
+  const bool far_cands = frame_tiles - 1 > TRA_PAIR_WINDOW;
+  const int reach = far_cands ? frame_tiles + 1 : TRA_PAIR_WINDOW;           // largest candidate offset
+  auto cand_offset = [&](int c) { return c < TRA_PAIR_WINDOW ? 1 + c : frame_tiles - 1 + (c - TRA_PAIR_WINDOW); };
+  const int win_rows = TRA_PAIR_CHUNK + reach;
   uint32_t* s_win = s_pair;                                                  // [win_rows][words]
-  uint16_t* s_band = (uint16_t*)(s_win + win_rows * words);                  // [NT][window]
+  uint16_t* s_band = (uint16_t*)(s_win + win_rows * words);                  // [NT][TRA_PAIR_CANDS]
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const long long bh = blockIdx.x;
   const uint8_t* mask_h = block_mask + bh * NB * (long long)NB;
   int32_t* out = pairs + bh * ((NT + 1) / 2) * 2;
 
+  // The window is a ring: the bitmap of tile t sits in row t % win_rows.  A chunk needs the tiles
+  // chunk0 .. chunk0 + TRA_PAIR_CHUNK - 1 + reach; all but the last TRA_PAIR_CHUNK are there already.
   for (int chunk0 = 0; chunk0 < NT; chunk0 += TRA_PAIR_CHUNK) {
-    const int rows = min(win_rows, NT - chunk0);
-    __syncthreads();                         // the previous chunk's window has been read
-    // one warp per window row; the loads of TRA_PAIR_LOADS words of the row are in flight together.
-    // The last rows of a window are the first rows of the next: they are moved, not read again.
-    const int keep = chunk0 > 0 ? TRA_PAIR_WINDOW : 0;
-    if (keep) {
-      for (int i = tid; i < keep * words; i += TRA_PAIR_THREADS) s_win[i] = s_win[TRA_PAIR_CHUNK * words + i];
-      __syncthreads();
-    }
-    for (int r = keep + warp; r < rows; r += TRA_PAIR_THREADS / 32) {
+    const int t_begin = chunk0 > 0 ? chunk0 + reach : 0, t_end = min(NT, chunk0 + win_rows);
+    __syncthreads();                         // the previous chunk's readers are done with the rows replaced now
+    // one warp per tile; the loads of TRA_PAIR_LOADS words of a mask row are in flight together
+    for (int t = t_begin + warp; t < t_end; t += TRA_PAIR_THREADS / 32) {
+      uint32_t* dst = s_win + (t % win_rows) * words;
       for (int wd0 = 0; wd0 < words; wd0 += TRA_PAIR_LOADS) {
         uint32_t on[TRA_PAIR_LOADS];
 #pragma unroll
         for (int q = 0; q < TRA_PAIR_LOADS; ++q) on[q] = 0u;
         for (int g = 0; g < G; ++g) {
-          const int u = (chunk0 + r) * G + g;
+          const int u = t * G + g;
           if (u >= NB) break;
           const uint8_t* row = mask_h + (long long)u * NB;
+          uint32_t got[TRA_PAIR_LOADS];
 #pragma unroll
-          for (int q = 0; q < TRA_PAIR_LOADS; ++q) {           // independent loads
-            const int j = (wd0 + q) * 32 + lane;
-            on[q] |= j < NB ? (uint32_t)row[j] : 0u;
-          }
+          for (int q = 0; q < TRA_PAIR_LOADS; ++q)             // independent loads (past the row: its last byte)
+            got[q] = __ldg(row + min((wd0 + q) * 32 + lane, NB - 1));
+#pragma unroll
+          for (int q = 0; q < TRA_PAIR_LOADS; ++q) on[q] |= got[q];
         }
 #pragma unroll
         for (int q = 0; q < TRA_PAIR_LOADS; ++q) {
-          const uint32_t bits = __ballot_sync(0xffffffffu, on[q] != 0u);
-          if (lane == 0 && wd0 + q < words) s_win[r * words + wd0 + q] = bits;
+          const uint32_t bits = __ballot_sync(0xffffffffu, on[q] != 0u && (wd0 + q) * 32 + lane < NB);
+          if (lane == 0 && wd0 + q < words) dst[wd0 + q] = bits;
         }
       }
     }
     __syncthreads();
-    for (int task = tid; task < TRA_PAIR_CHUNK * TRA_PAIR_WINDOW; task += TRA_PAIR_THREADS) {
-      const int ul = task / TRA_PAIR_WINDOW, c = task - ul * TRA_PAIR_WINDOW;
-      const int u = chunk0 + ul, v = u + 1 + c;
+    for (int task = tid; task < TRA_PAIR_CHUNK * TRA_PAIR_CANDS; task += TRA_PAIR_THREADS) {
+      const int ul = task / TRA_PAIR_CANDS, c = task - ul * TRA_PAIR_CANDS;
+      const int u = chunk0 + ul, v = u + cand_offset(c);
       if (u >= NT) continue;
       uint32_t d = 0xffffu;
-      if (v < NT) {
+      if (v < NT && (c < TRA_PAIR_WINDOW || far_cands)) {
         d = 0;
-        const uint32_t* a = s_win + ul * words;
-        const uint32_t* b = s_win + (ul + 1 + c) * words;
+        const uint32_t* a = s_win + (u % win_rows) * words;
+        const uint32_t* b = s_win + (v % win_rows) * words;
         for (int wd = 0; wd < words; ++wd) d += __popc(a[wd] ^ b[wd]);
         d = min(d, 0xfffeu);
       }
-      s_band[u * TRA_PAIR_WINDOW + c] = (uint16_t)d;
+      s_band[u * TRA_PAIR_CANDS + c] = (uint16_t)d;
     }
   }
   __syncthreads();
@@ -498,16 +503,19 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
   };
   int n_out = 0;
   for (int u = first_free_from(0); u < NT; u = first_free_from(u + 1)) {
-    const int vc = min(u + 1 + lane, NT - 1);
+    const int vo = u + cand_offset(min(lane, TRA_PAIR_CANDS - 1));
+    const int vc = min(vo, NT - 1);
     const unsigned long long w = __shfl_sync(0xffffffffu, used, vc >> 6);
-    uint32_t key = 0xffffffffu;              // (unshared blocks, window position) of this lane's candidate
-    if (lane < TRA_PAIR_WINDOW && u + 1 + lane < NT && !((w >> (vc & 63)) & 1ull))
-      key = ((uint32_t)s_band[u * TRA_PAIR_WINDOW + lane] << 8) | (uint32_t)lane;
+    uint32_t key = 0xffffffffu;              // (unshared blocks, candidate number) of this lane's candidate
+    if (lane < TRA_PAIR_CANDS && vo < NT && !((w >> (vc & 63)) & 1ull)) {
+      const uint32_t d = s_band[u * TRA_PAIR_CANDS + lane];
+      if (d != 0xffffu) key = (d << 8) | (uint32_t)lane;
+    }
     key = __reduce_min_sync(0xffffffffu, key);
     int v;
     if (key != 0xffffffffu) {
-      v = u + 1 + (int)(key & 0xffu);
-    } else {                                 // nothing left in the window: the next unmatched tile, if any
+      v = u + cand_offset((int)(key & 0xffu));
+    } else {                                 // no candidate left: the next unmatched tile after the window, if any
       mark(u);
       v = first_free_from(u + 1 + TRA_PAIR_WINDOW);
       if (v >= NT) v = -1;
@@ -561,14 +569,18 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     const int b = plan->cfg.block;
     const int G = (128 % b == 0) ? 128 / b : 1;
     const int NT = (NB + G - 1) / G;
-    const size_t pair_smem = ((size_t)(TRA_PAIR_CHUNK + TRA_PAIR_WINDOW) * ((NB + 31) / 32)) * 4 +
-                             (size_t)NT * TRA_PAIR_WINDOW * 2;
+    // tiles per frame, rounded: the tile one frame ahead of u is u + frame_tiles or a neighbour of it
+    const long long tile_tokens = (long long)b * G;
+    const int frame_tiles = (int)(((long long)plan->cfg.H * plan->cfg.W + tile_tokens / 2) / tile_tokens);
+    const int reach = frame_tiles - 1 > TRA_PAIR_WINDOW ? frame_tiles + 1 : TRA_PAIR_WINDOW;
+    const size_t pair_smem = ((size_t)(TRA_PAIR_CHUNK + reach) * ((NB + 31) / 32)) * 4 +
+                             (size_t)NT * TRA_PAIR_CANDS * 2;
     if (pair_smem > 200 * 1024 || NT > 2048) return TRA_ERR_UNSUPPORTED;
     if (pair_smem > 48 * 1024)
       TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)pair_smem));
     tra_pair_tiles_kernel<<<(unsigned)BH, TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G,
-                                                                                 plan->d_status);
+                                                                                 frame_tiles, plan->d_status);
     TRA_CUDA_CHECK(cudaGetLastError());
   }
   return TRA_OK;
