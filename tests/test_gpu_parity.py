@@ -367,6 +367,49 @@ def test_sparse_attn_all_rows(cfg, kind):
     plan.close()
 
 
+CFG_FRAMES128 = common.small_config(5, 32, 48, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16, seed=84,
+                                    s_lo=0.2, s_hi=5.0)      # 12 query tiles per frame
+
+
+@pytest.mark.parametrize("cfg,n_text,gamma", [(CFG_TINY, 0, None), (CFG_RAGGED64, 50, None), (CFG_D128_B64, 0, None),
+                                              (CFG_MID128, 0, None), (CFG_FRAMES128, 0, None),
+                                              (CFG_FRAMES128, 100, 0.05)],
+                         ids=["tiny", "ragged64+text", "d128_b64", "mid128", "frames128", "frames128+text-slow-decay"])
+def test_tile_pair_table(cfg, n_text, gamma):
+    """The tile-pair table of the block-mask call: every 128-row query tile appears exactly once, and
+    the sparse launch gives the same bits with it as with consecutive tiles (plain and with the token
+    mask).  The last two shapes have more tiles per frame than the pairing window, so tiles one frame
+    ahead are candidates too."""
+    if gamma is not None:
+        cfg = dict(cfg, gamma=gamma)
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg, n_text=n_text)
+    S = geo.N + n_text
+    heads = cfg["heads"]
+    Qr, Kr, Vr = workloads.make_qkv(cfg, DEV)
+    if n_text:
+        Qr, Kr, Vr = workloads.append_text(Qr, Kr, Vr, cfg, n_text)
+    Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    _, H, _ = plan.entropy_attn(Q, K, V)
+    _, _, ridx = plan.budget_radius(H)
+    mask, row_ptr, col_idx, nnz, pairs = plan.build_block_mask(ridx, want_tile_pairs=True)
+    plan.check_status()
+    n_tiles = (S + 127) // 128 if 128 % geo.block == 0 else (S + geo.block - 1) // geo.block
+    p = pairs.reshape(heads, -1, 2).cpu().numpy()
+    assert p.shape[1] == (n_tiles + 1) // 2
+    for h in range(heads):
+        assert np.array_equal(np.sort(p[h][p[h] >= 0]), np.arange(n_tiles))
+        assert (p[h][:, 0] >= 0).all()                               # only the second slot may be empty
+    O1, lse1 = plan.sparse_attn(Q, K, V, row_ptr, col_idx, tile_pairs=pairs, want_lse=True)
+    O2, lse2 = plan.sparse_attn(Q, K, V, row_ptr, col_idx, want_lse=True)
+    assert torch.equal(O1, O2) and torch.equal(lse1, lse2)
+    T1, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx, tile_pairs=pairs)
+    T2, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx)
+    plan.check_status()
+    assert torch.equal(T1, T2)
+    plan.close()
+
+
 @pytest.mark.parametrize("cfg,n_text", [(CFG_TINY, 0), (CFG_RAGGED64, 0), (CFG_RAGGED128, 0), (CFG_MID128, 0),
                                         (CFG_RAGGED64, 50), (CFG_RAGGED128, 200)],
                          ids=["tiny", "ragged64", "ragged128", "mid128", "ragged64+text", "ragged128+text"])
