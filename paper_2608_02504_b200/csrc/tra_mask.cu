@@ -401,8 +401,8 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 // ---------------------------------------------------------------------------------------
 // Tile pairing for the block-sparse attention launch.  That launch gives every CTA two 128-row
 // query tiles which walk the union of their key-block lists; a key block only one of the two
-// retains leaves the other tile idle.  This kernel pairs tiles with similar lists: one CTA per
-// (batch, head); tile t covers the query blocks [t G, (t + 1) G), G = 128 / block.
+// retains leaves the other tile idle.  This kernel pairs tiles with similar lists, per (batch,
+// head); tile t covers the query blocks [t G, (t + 1) G), G = 128 / block.
 //   1. row bitmaps of a window of tiles are built in shared memory (ballots over the byte mask),
 //      and for every tile u the number of key blocks that u and each of its candidates do not
 //      share is stored.  The candidates are the next TRA_PAIR_WINDOW tiles and, when a frame holds
@@ -410,7 +410,8 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 //      frame: with a slow temporal decay those share far more key blocks than spatial neighbours);
 //   2. one warp matches the tiles greedily in ascending order: the first unmatched tile takes the
 //      unmatched candidate with the fewest unshared key blocks, or, when none is left, the next
-//      unmatched tile after the window.  Every tile is matched (one is left alone
+//      unmatched tile after the window.
+// Four CTAs per (batch, head) take a quarter of the tiles each and match inside it.  Every tile is matched (one is left alone
 //      when their number is odd): pairs[i] = (u, v) for i < ceil(NT / 2), v = -1 for a lone tile.
 // Any perfect matching gives the same attention output; the choice only moves time.
 // ---------------------------------------------------------------------------------------
@@ -437,10 +438,16 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
   const uint8_t* mask_h = block_mask + bh * NB * (long long)NB;
   int32_t* out = pairs + bh * ((NT + 1) / 2) * 2;
 
+  // This CTA's quarter of the tiles (an even number of them, so only the last quarter can leave a
+  // tile alone); candidates stay inside the quarter.
+  const int seg_len = ((NT + 3) / 4 + 1) & ~1;
+  const int seg_begin = (int)blockIdx.y * seg_len, seg_end = min(NT, seg_begin + seg_len);
+  if (seg_begin >= seg_end) return;
+
   // The window is a ring: the bitmap of tile t sits in row t % win_rows.  A chunk needs the tiles
   // chunk0 .. chunk0 + TRA_PAIR_CHUNK - 1 + reach; all but the last TRA_PAIR_CHUNK are there already.
-  for (int chunk0 = 0; chunk0 < NT; chunk0 += TRA_PAIR_CHUNK) {
-    const int t_begin = chunk0 > 0 ? chunk0 + reach : 0, t_end = min(NT, chunk0 + win_rows);
+  for (int chunk0 = seg_begin; chunk0 < seg_end; chunk0 += TRA_PAIR_CHUNK) {
+    const int t_begin = chunk0 > seg_begin ? chunk0 + reach : seg_begin, t_end = min(seg_end, chunk0 + win_rows);
     __syncthreads();                         // the previous chunk's readers are done with the rows replaced now
     // one warp per tile; the loads of TRA_PAIR_LOADS words of a mask row are in flight together
     for (int t = t_begin + warp; t < t_end; t += TRA_PAIR_THREADS / 32) {
@@ -471,44 +478,44 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
     for (int task = tid; task < TRA_PAIR_CHUNK * TRA_PAIR_CANDS; task += TRA_PAIR_THREADS) {
       const int ul = task / TRA_PAIR_CANDS, c = task - ul * TRA_PAIR_CANDS;
       const int u = chunk0 + ul, v = u + cand_offset(c);
-      if (u >= NT) continue;
+      if (u >= seg_end) continue;
       uint32_t d = 0xffffu;
-      if (v < NT && (c < TRA_PAIR_WINDOW || far_cands)) {
+      if (v < seg_end && (c < TRA_PAIR_WINDOW || far_cands)) {
         d = 0;
         const uint32_t* a = s_win + (u % win_rows) * words;
         const uint32_t* b = s_win + (v % win_rows) * words;
         for (int wd = 0; wd < words; ++wd) d += __popc(a[wd] ^ b[wd]);
         d = min(d, 0xfffeu);
       }
-      s_band[u * TRA_PAIR_CANDS + c] = (uint16_t)d;
+      s_band[(u - seg_begin) * TRA_PAIR_CANDS + c] = (uint16_t)d;
     }
   }
   __syncthreads();
-  if (warp != 0) return;
   // Greedy matching by one warp.  The "matched" flags of all tiles live in registers: lane l holds the
   // 64 tiles [64 l, 64 l + 64) (NT <= 2048), so a step costs a few shuffles and no shared-memory round trip.
+  if (warp != 0) return;
   unsigned long long used = 0ull;
-  auto first_free_from = [&](int from) -> int {          // the first unmatched tile >= from, or NT
+  auto first_free_from = [&](int from) -> int {          // the first unmatched tile in [from, seg_end), or seg_end
     unsigned long long free_bits = ~used;
     const int lo = 64 * lane;
     if (lo + 63 < from) free_bits = 0ull;
     else if (lo < from) free_bits &= ~0ull << (from - lo);
-    if (lo >= NT) free_bits = 0ull;
-    else if (NT - lo < 64) free_bits &= (1ull << (NT - lo)) - 1ull;
-    const uint32_t cand = free_bits ? (uint32_t)(lo + __ffsll((long long)free_bits) - 1) : (uint32_t)NT;
+    if (lo >= seg_end) free_bits = 0ull;
+    else if (seg_end - lo < 64) free_bits &= (1ull << (seg_end - lo)) - 1ull;
+    const uint32_t cand = free_bits ? (uint32_t)(lo + __ffsll((long long)free_bits) - 1) : (uint32_t)seg_end;
     return (int)__reduce_min_sync(0xffffffffu, cand);
   };
   auto mark = [&](int t) {
     if (t >= 0 && lane == (t >> 6)) used |= 1ull << (t & 63);
   };
-  int n_out = 0;
-  for (int u = first_free_from(0); u < NT; u = first_free_from(u + 1)) {
+  int n_out = seg_begin / 2;
+  for (int u = first_free_from(seg_begin); u < seg_end; u = first_free_from(u + 1)) {
     const int vo = u + cand_offset(min(lane, TRA_PAIR_CANDS - 1));
-    const int vc = min(vo, NT - 1);
+    const int vc = min(vo, seg_end - 1);
     const unsigned long long w = __shfl_sync(0xffffffffu, used, vc >> 6);
     uint32_t key = 0xffffffffu;              // (unshared blocks, candidate number) of this lane's candidate
-    if (lane < TRA_PAIR_CANDS && vo < NT && !((w >> (vc & 63)) & 1ull)) {
-      const uint32_t d = s_band[u * TRA_PAIR_CANDS + lane];
+    if (lane < TRA_PAIR_CANDS && vo < seg_end && !((w >> (vc & 63)) & 1ull)) {
+      const uint32_t d = s_band[(u - seg_begin) * TRA_PAIR_CANDS + lane];
       if (d != 0xffffu) key = (d << 8) | (uint32_t)lane;
     }
     key = __reduce_min_sync(0xffffffffu, key);
@@ -518,7 +525,7 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
     } else {                                 // no candidate left: the next unmatched tile after the window, if any
       mark(u);
       v = first_free_from(u + 1 + TRA_PAIR_WINDOW);
-      if (v >= NT) v = -1;
+      if (v >= seg_end) v = -1;
     }
     mark(u);
     mark(v);
@@ -579,7 +586,7 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     if (pair_smem > 48 * 1024)
       TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)pair_smem));
-    tra_pair_tiles_kernel<<<(unsigned)BH, TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G,
+    tra_pair_tiles_kernel<<<dim3((unsigned)BH, 4), TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G,
                                                                                  frame_tiles, plan->d_status);
     TRA_CUDA_CHECK(cudaGetLastError());
   }
