@@ -1,4 +1,6 @@
 // Block-mask construction from per-query radii (Algorithm 1) and its CSR active-block list.
+#include <algorithm>
+
 #include "tra_common.cuh"
 
 #define TRA_MASK_THREADS 128
@@ -51,9 +53,6 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
                       int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal,
                       int* __restrict__ status) {
   extern __shared__ int32_t s_dyn[];
-  __shared__ __align__(16) int s_rank_key[128];
-  __shared__ uint32_t s_sorted[128];        // queries in descending candidate index: coord | 0, and ...
-  __shared__ uint16_t s_sorted_r[128];      // ... their candidate index
   __shared__ tra_block_boxes_t s_ubox;
   __shared__ int s_rstar, s_count, s_whole[2];
 
@@ -64,13 +63,17 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   int32_t* s_frame_ylo = s_dyn + Tp;                               // [T] rows of the frame that hold keys of an
   int32_t* s_frame_yhi = s_dyn + 2 * Tp;                           // [T] undecided key block (yhi < 0: none)
   int32_t* s_diff = s_dyn + 3 * Tp;                                // [H][Wp]
-  uint32_t* s_cols = (uint32_t*)(s_diff + n_diff);                 // [NB] reached columns | high columns << 16
-  uint8_t* s_state = (uint8_t*)(s_cols + NB);                      // [NB] 0 / 1 decided, 2 undecided
+  uint32_t* s_cols = (uint32_t*)(s_diff + n_diff);                 // [NB] reached columns | high columns << 16 |
+                                                                   // state << 30 (0 / 1 decided, 2 undecided)
   const int HW = H * W;
   const int n_pos = kQuads ? HW / 4 : HW;                          // entries of the position table
-  uint32_t* s_cnt = (uint32_t*)(s_dyn + 3 * Tp + n_diff + (5 * NB + 15) / 16 * 4);   // [H * W] bytes (16-byte
+  uint32_t* s_cnt = (uint32_t*)(s_dyn + 3 * Tp + n_diff + (NB + 3) / 4 * 4);   // [max(H * W, 1280)] bytes (16-byte
                                                                    // aligned): counts in tile-major order
-  uint16_t* s_pos = (uint16_t*)(s_cnt + (HW + 15) / 16 * 4);       // [n_pos] the plan's position table
+  uint16_t* s_pos = (uint16_t*)(s_cnt + (max(HW, 1280) + 15) / 16 * 4);   // [n_pos] the plan's position table
+  // the sort of the queries by candidate index is over before the first counts are written
+  int* s_rank_key = (int*)s_cnt;                                   // [128]
+  uint32_t* s_sorted = s_cnt + 128;         // [128] queries in descending candidate index: coord, and ...
+  uint16_t* s_sorted_r = (uint16_t*)(s_cnt + 256);                 // [128] ... their candidate index
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x;
@@ -115,9 +118,6 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   for (int i = tid; i < T; i += TRA_MASK_THREADS) {
     s_frame_ylo[i] = H;
     s_frame_yhi[i] = -1;
-  }
-  for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
-    s_cols[v] = 0;
   }
   __syncthreads();
 
@@ -176,11 +176,12 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
           if (s_theta_star[dt_min] >= gy * gy + gx * gx) all_reject = false;
           if (s_theta_star[dt_max] < fy * fy + fx * fx) all_accept = false;
         }
+        if (!all_reject && !all_accept) break;     // undecided whatever the other boxes say
       }
       decided = all_reject ? 0 : (all_accept ? 1 : 2);
     }
     if (keep_diagonal && v == u) decided = 1;
-    s_state[v] = (uint8_t)decided;
+    s_cols[v] = (uint32_t)decided << 30;
     if (decided == 2) {
       // frames this key block has tokens in, and the rows of each that hold them
       for (int iv = 0; iv < vb.n_box; ++iv)
@@ -276,7 +277,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     const int p_begin = f * HW, p_end = min(N, (f + 1) * HW);
     const int v_first = p_begin / b, v_last = (p_end - 1) / b;     // video blocks only: p_end <= N
     for (int v = v_first + warp; v <= v_last; v += TRA_MASK_WARPS) {
-      if (s_state[v] != 2) continue;
+      if ((s_cols[v] >> 30) != 2u) continue;
       const int i0 = max(v * b, p_begin) - p_begin, i1 = min((v + 1) * b, p_end) - p_begin;   // bytes [i0, i1)
       int acc = 0;                                        // reached | high << 16 of this lane's keys
       if (((i0 | i1) & 3) == 0 && i1 - i0 == 128) {       // 32 whole words, one per lane (uniform across the warp)
@@ -326,8 +327,9 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   __syncthreads();
   kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
-    if (s_state[v] != 2) continue;
-    const int ne = (int)(s_cols[v] & 0xffffu), hi = (int)(s_cols[v] >> 16);
+    const uint32_t cv = s_cols[v];
+    if ((cv >> 30) != 2u) continue;
+    const int ne = (int)(cv & 0xffffu), hi = (int)((cv >> 16) & 0x3fffu);
     const int keep = (ne > 0) && (10 * hi > 6 * ne);
     mask_row[v] = (uint8_t)keep;
     kept += keep;
@@ -552,7 +554,7 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
 
   const int H = plan->cfg.H, W = plan->cfg.W;
   size_t smem = ((size_t)3 * ((T + 3) & ~3) + (size_t)H * tra_field_row_words(W)) * sizeof(int32_t) +
-                ((size_t)NB * 5 + 15) / 16 * 16 + ((size_t)H * W + 15) / 16 * 16 +
+                ((size_t)NB + 3) / 4 * 16 + (std::max<size_t>((size_t)H * W, 1280) + 15) / 16 * 16 +
                 ((((size_t)H * W / (plan->field_quads ? 4 : 1)) + 7) & ~(size_t)7) * sizeof(uint16_t);
   if (smem > 200 * 1024 || !plan->d_field_pos) return TRA_ERR_UNSUPPORTED;   // frame too large for the count field
   dim3 grid((unsigned)NB, (unsigned)BH);
