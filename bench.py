@@ -613,7 +613,7 @@ def run_workload(api, name, dev, peak_tf, reps=2, gamma=None):
     return out
 
 
-def run_e2e(args, api, plan, src_dev, O_raster, flops_rank, world, dev, group=8, first_group=2):
+def run_e2e(args, api, plan, src_dev, O_raster, flops_rank, world, dev, group=8, first_group=1):
     """Same pass with Q, K, V in pinned host memory and O read back to pinned host memory, through
     the library's host pipeline: groups of `group` heads (a smaller first group, so the kernels
     start early), the copies of neighbouring groups overlapping the kernels of the current one.

@@ -198,9 +198,10 @@ int tra_sparse_attn(const tra_plan_t* plan, const void* Q, const void* K, const 
  * mask, block-sparse attention (retained blocks in full), layout back — over
  *   Q_host, K_host, V_host : HOST pointers, bf16 [heads, S, head_dim], RASTER token order (read),
  *   O_host                 : HOST pointer, same shape and order (written): the block-sparse output.
- * Heads are independent problems, so the pass runs in groups of `group` heads (the first group
- * holds `first_group` <= group heads, so that the kernels start early, and the last group is split
- * so that little output is left to copy after the last kernel); the host-to-device copy of
+ * Heads are independent problems, so the pass runs in groups of at most `group` heads (the first
+ * group holds `first_group` <= group heads, so that the kernels start early, the following ones
+ * twice as many as the one before until `group` is reached, and the last group is split so that
+ * little output is left to copy after the last kernel); the host-to-device copy of
  * the next group and the device-to-host copy of the previous one run on two copy streams owned by
  * the plan while the kernels of the current group run on `stream`.  Pinned (page-locked) host
  * memory is needed for the copies to overlap; pageable memory works but serialises.

@@ -318,14 +318,16 @@ class HostPipeline:
 
     @staticmethod
     def group_sizes(heads, group, first_group):
-        """The head groups of one pass (mirrors the library): a small first and a small last group."""
-        sizes, left = [], heads
+        """The head groups of one pass (mirrors the library): a small first group, doubling up to
+        ``group``, and a small last group."""
+        sizes, left, ramp = [], heads, first_group
         while left > 0:
-            n = min(first_group if not sizes else group, left)
+            n = min(ramp, left)
             if left - n == 0 and n > first_group and sizes:
                 n -= first_group
             sizes.append(n)
             left -= n
+            ramp = min(2 * ramp, group)
         return sizes
 
     @staticmethod

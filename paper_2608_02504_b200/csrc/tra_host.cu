@@ -118,11 +118,12 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
 
   cudaEvent_t in_free[2] = {nullptr, nullptr};    // the gathers that read staging buffer b are done
   cudaEvent_t out_free[2] = {nullptr, nullptr};   // the copy out of output buffer b is done
-  // group sizes: a small first group (the kernels start early) and a small last one (little output
-  // left to copy after the last kernel)
+  // group sizes: a small first group (the kernels start early), doubling up to `group` (a group's
+  // kernels cover the copy of the next, twice as large), and a small last one (little output left to
+  // copy after the last kernel)
   std::vector<int> sizes;
-  for (int left = heads; left > 0;) {
-    int n = std::min(sizes.empty() ? first_group : group, left);
+  for (int left = heads, ramp = first_group; left > 0; ramp = std::min(2 * ramp, group)) {
+    int n = std::min(ramp, left);
     if (left - n == 0 && n > first_group && !sizes.empty()) n -= first_group;   // split the last group
     sizes.push_back(n);
     left -= n;
