@@ -761,7 +761,7 @@ def main():
     ap.add_argument("--tau", type=float, default=None)
     ap.add_argument("--heads", type=int, default=None, help="override the head count (profiling on a small case)")
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-rows", type=int, default=2048)
+    ap.add_argument("--cpu-rows", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="the timed steps, e2e and CPU baseline only")
     ap.add_argument("--no-schedule", dest="schedule", action="store_false")
