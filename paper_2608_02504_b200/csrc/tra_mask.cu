@@ -32,8 +32,9 @@
 //    stores the counts as bytes in the frame's tile-major order, so that the keys of a block are
 //    consecutive bytes.  Every undecided key block then reads the counts of its own keys in that
 //    frame (c_j by definition), four per 32-bit word, and compares all four with the two
-//    thresholds at once (adding 127 - t to a byte sets its top bit iff the byte exceeds t).  When the query block lies in one frame t0 the
-//    frames t0 - k and t0 + k see the same thresholds, so one field serves both.
+//    thresholds at once (adding 127 - t to a byte sets its top bit iff the byte exceeds t).  When
+//    the query block lies in one frame t0 the frames t0 - k and t0 + k see the same thresholds,
+//    so one field serves both.
 // The outcome equals the unpruned vote bit for bit.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ int tra_isqrt_small(int n) {
@@ -49,9 +50,9 @@ template <bool kQuads>
 __global__ void __launch_bounds__(TRA_MASK_THREADS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
-                      const uint16_t* __restrict__ field_pos, uint8_t* __restrict__ block_mask, int32_t* __restrict__ row_ptr, int N, int S, int NB,
-                      int NBv, int b, int T, int H, int W, int n_radii, int keep_diagonal,
-                      int* __restrict__ status) {
+                      const uint16_t* __restrict__ field_pos, uint8_t* __restrict__ block_mask,
+                      int32_t* __restrict__ row_ptr, int N, int S, int NB, int NBv, int b, int T, int H, int W,
+                      int n_radii, int keep_diagonal, int* __restrict__ status) {
   extern __shared__ int32_t s_dyn[];
   __shared__ tra_block_boxes_t s_ubox;
   __shared__ int s_rstar, s_count, s_whole[2];
@@ -562,8 +563,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   if (smem > 48 * 1024)
     TRA_CUDA_CHECK(cudaFuncSetAttribute(vote, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   vote<<<grid, TRA_MASK_THREADS, smem, stream>>>(
-      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, plan->d_field_pos, block_mask, row_ptr, plan->N, plan->S,
-      NB, plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0,
+      ridx, plan->d_coord_packed, plan->d_theta, plan->d_boxes, plan->d_field_pos, block_mask, row_ptr, plan->N,
+      plan->S, NB, plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0,
       plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,
