@@ -414,8 +414,9 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 //   2. one warp matches the tiles greedily in ascending order: the first unmatched tile takes the
 //      unmatched candidate with the fewest unshared key blocks, or, when none is left, the next
 //      unmatched tile after the window.
-// Four CTAs per (batch, head) take a quarter of the tiles each and match inside it.  Every tile is matched (one is left alone
-//      when their number is odd): pairs[i] = (u, v) for i < ceil(NT / 2), v = -1 for a lone tile.
+// Four CTAs per (batch, head) take a quarter of the tiles each and match inside it.  Every tile is
+// matched (one is left alone when their number is odd): pairs[i] = (u, v) for i < ceil(NT / 2),
+// v = -1 for a lone tile.
 // Any perfect matching gives the same attention output; the choice only moves time.
 // ---------------------------------------------------------------------------------------
 #define TRA_PAIR_WINDOW 8
@@ -589,8 +590,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     if (pair_smem > 48 * 1024)
       TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)pair_smem));
-    tra_pair_tiles_kernel<<<dim3((unsigned)BH, 4), TRA_PAIR_THREADS, pair_smem, stream>>>(block_mask, tile_pairs, NB, NT, G,
-                                                                                 frame_tiles, plan->d_status);
+    tra_pair_tiles_kernel<<<dim3((unsigned)BH, 4), TRA_PAIR_THREADS, pair_smem, stream>>>(
+        block_mask, tile_pairs, NB, NT, G, frame_tiles, plan->d_status);
     TRA_CUDA_CHECK(cudaGetLastError());
   }
   return TRA_OK;
