@@ -27,6 +27,7 @@ struct tra_plan {
   int N, NB, n_radii;   // N = T*H*W video tokens; NB = blocks of the whole sequence
   int S, NBv;           // S = N + n_text tokens in the sequence; NBv = video blocks (see tra_plan_create)
   int device;
+  int sm_count;         // multiprocessors of the device
   double z_tau;       // Phi^-1(tau), for the lognormal budget map
   // host copies
   double* h_radii;

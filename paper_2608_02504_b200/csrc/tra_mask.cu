@@ -414,7 +414,8 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 //   2. one warp matches the tiles greedily in ascending order: the first unmatched tile takes the
 //      unmatched candidate with the fewest unshared key blocks, or, when none is left, the next
 //      unmatched tile after the window.
-// Four CTAs per (batch, head) take a quarter of the tiles each and match inside it.  Every tile is
+// Up to four CTAs per (batch, head), as many as fit the device in one wave, take a part of the tiles
+// each and match inside it.  Every tile is
 // matched (one is left alone when their number is odd): pairs[i] = (u, v) for i < ceil(NT / 2),
 // v = -1 for a lone tile.
 // Any perfect matching gives the same attention output; the choice only moves time.
@@ -442,9 +443,10 @@ tra_pair_tiles_kernel(const uint8_t* __restrict__ block_mask, int32_t* __restric
   const uint8_t* mask_h = block_mask + bh * NB * (long long)NB;
   int32_t* out = pairs + bh * ((NT + 1) / 2) * 2;
 
-  // This CTA's quarter of the tiles (an even number of them, so only the last quarter can leave a
-  // tile alone); candidates stay inside the quarter.
-  const int seg_len = ((NT + 3) / 4 + 1) & ~1;
+  // This CTA's part of the tiles (gridDim.y parts of an even number of tiles, so only the last part
+  // can leave a tile alone); candidates stay inside the part.
+  const int n_seg = (int)gridDim.y;
+  const int seg_len = ((NT + n_seg - 1) / n_seg + 1) & ~1;
   const int seg_begin = (int)blockIdx.y * seg_len, seg_end = min(NT, seg_begin + seg_len);
   if (seg_begin >= seg_end) return;
 
@@ -590,7 +592,8 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     if (pair_smem > 48 * 1024)
       TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)pair_smem));
-    tra_pair_tiles_kernel<<<dim3((unsigned)BH, 4), TRA_PAIR_THREADS, pair_smem, stream>>>(
+    const unsigned n_seg = (unsigned)std::max(1ll, std::min(4ll, (long long)plan->sm_count / BH));   // one CTA per SM
+    tra_pair_tiles_kernel<<<dim3((unsigned)BH, n_seg), TRA_PAIR_THREADS, pair_smem, stream>>>(
         block_mask, tile_pairs, NB, NT, G, frame_tiles, plan->d_status);
     TRA_CUDA_CHECK(cudaGetLastError());
   }

@@ -142,7 +142,8 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   // kept dense like a text block, so that every text key stays visible: Section 3.2, last paragraph)
   p->NBv = cfg->n_text > 0 ? p->N / cfg->block : (p->N + cfg->block - 1) / cfg->block;
   p->z_tau = tra_inverse_normal_cdf(cfg->tau);
-  if (cudaGetDevice(&p->device) != cudaSuccess) {
+  if (cudaGetDevice(&p->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) != cudaSuccess) {
     delete p;
     return TRA_ERR_CUDA;
   }
