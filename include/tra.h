@@ -164,7 +164,9 @@ int tra_budget_radius(const tra_plan_t* plan, const float* entropy, int32_t* bud
  *               no counterpart: tra_sparse_attn gives each thread block two 128-row query tiles that
  *               share the key/value tiles they both retain, and this table pairs tiles whose block
  *               lists are similar (entry -1 = no second tile).  Pass it to tra_sparse_attn together
- *               with row_ptr / col_idx; it changes the speed of that call, never its result. */
+ *               with row_ptr / col_idx; it changes the speed of that call, never its result.
+ *               Block sizes that do not divide 128 have no attention launch and no query tiles:
+ *               with such a plan a non-NULL tile_pairs returns TRA_ERR_UNSUPPORTED (nothing is run). */
 int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* block_mask,
                          int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
                          int64_t* nnz_out, int32_t* tile_pairs, int B, int heads, void* stream);

@@ -17,6 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("TRA_B200_LIB") or os.path.join(_HERE, "libtra_b200.so")
 
 TRA_OK = 0
+TRA_ERR_INVALID_ARG, TRA_ERR_UNSUPPORTED, TRA_ERR_CAPACITY, TRA_ERR_CUDA, TRA_ERR_TIMEOUT, TRA_ERR_BOUNDS = -1, -2, -3, -4, -5, -6
 TRA_KEEP_DIAGONAL = 1
 TRA_RADII_EXTENDED = 0
 TRA_RADII_LITERAL = 1

@@ -554,6 +554,7 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   const int NB = plan->NB, T = plan->cfg.T;
   const long long BH = (long long)B * heads;
   if (NB > 65535 || BH > 65535) return TRA_ERR_UNSUPPORTED;
+  if (tile_pairs && 128 % plan->cfg.block != 0) return TRA_ERR_UNSUPPORTED;   // no attention launch, no query tiles
   const long long rows = BH * NB;
 
   const int H = plan->cfg.H, W = plan->cfg.W;
@@ -577,10 +578,9 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
       block_mask, row_ptr, col_idx, rows, NB, (long long)col_idx_capacity, plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   if (tile_pairs) {
-    // query tiles of the attention launch: 128 rows = G blocks (block sizes that do not divide 128
-    // have no attention kernel; their table pairs consecutive "tiles" of one block each)
+    // query tiles of the attention launch: 128 rows = G blocks
     const int b = plan->cfg.block;
-    const int G = (128 % b == 0) ? 128 / b : 1;
+    const int G = 128 / b;
     const int NT = (NB + G - 1) / G;
     // tiles per frame, rounded: the tile one frame ahead of u is u + frame_tiles or a neighbour of it
     const long long tile_tokens = (long long)b * G;

@@ -232,6 +232,31 @@ def test_random_geometries_integer_stages_and_token_mask(cfg):
     plan.close()
 
 
+@pytest.mark.parametrize("block", [48, 80])
+def test_block_sizes_that_do_not_divide_the_query_tile(block):
+    """Block sizes like the paper's 40 .. 120 have a block mask (bit for bit against the oracle) but no
+    attention launch, hence no query tiles to pair: asking for the tile-pair table is refused before
+    anything runs, and the mask buffers stay untouched."""
+    cfg = common.small_config(4, 12, 20, heads=2, head_dim=128, block=block, tile_h=4, tile_w=8, seed=85)
+    geo = common.oracle_geometry(cfg)
+    ridx = random_ridx(geo, cfg["heads"], np.random.default_rng(21), "entropy")
+    plan = make_plan(cfg)
+    mask, row_ptr, col_idx, nnz = run_mask(plan, ridx)
+    ref = np.stack([oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx[h]) for h in range(cfg["heads"])])
+    assert np.array_equal(mask, ref)
+    rp, ci = oracle.csr_from_block_mask(ref)
+    assert nnz == rp[-1] and np.array_equal(row_ptr.astype(np.int64), rp) and np.array_equal(col_idx[:nnz], ci)
+    ridx_t = torch.from_numpy(ridx.view(np.int16)).to(DEV)[None]
+    sentinel = torch.full((1, cfg["heads"], geo.NB, geo.NB), 7, dtype=torch.uint8, device=DEV)
+    with pytest.raises(api().TraError) as err:
+        plan.build_block_mask(ridx_t, block_mask=sentinel, want_tile_pairs=True)
+    assert err.value.code == api().TRA_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+    assert bool((sentinel == 7).all())
+    plan.check_status()
+    plan.close()
+
+
 def test_block_mask_capacity_error_is_reported():
     cfg = CFG_TINY
     geo = common.oracle_geometry(cfg)
