@@ -747,9 +747,11 @@ def test_batch_and_side_stream():
     Q, K, V = (torch.cat([a, b], dim=0).contiguous() for a, b in ((Q1, Q2), (K1, K2), (V1, V2)))
     O, H, _ = plan.entropy_attn(Q, K, V)
     _, _, ridx = plan.budget_radius(H)
-    mask, row_ptr, col_idx, nnz = plan.build_block_mask(ridx)
-    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)
+    mask, row_ptr, col_idx, nnz, pairs = plan.build_block_mask(ridx, want_tile_pairs=True)
+    Os, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, tile_pairs=pairs)      # the table is per (batch, head)
+    Ot, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx, tile_pairs=pairs)
     plan.check_status()
+    assert torch.equal(Os, plan.sparse_attn(Q, K, V, row_ptr, col_idx)[0])
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     for b, (q, k, v) in enumerate(((Q1, K1, V1), (Q2, K2, V2))):
@@ -758,10 +760,11 @@ def test_batch_and_side_stream():
             _, _, r = plan.budget_radius(h)
             m, rp, ci, nz = plan.build_block_mask(r)
             os_, _ = plan.sparse_attn(q, k, v, rp, ci)
+            ot_, _ = plan.sparse_attn(q, k, v, rp, ci, ridx=r)
         side.synchronize()
         assert torch.equal(o[0], O[b]) and torch.equal(h[0], H[b])
         assert torch.equal(r[0], ridx[b]) and torch.equal(m[0], mask[b])
-        assert torch.equal(os_[0], Os[b])
+        assert torch.equal(os_[0], Os[b]) and torch.equal(ot_[0], Ot[b])
     plan.check_status()
     plan.close()
 
