@@ -171,6 +171,33 @@ int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* 
                          int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
                          int64_t* nnz_out, int32_t* tile_pairs, int B, int heads, void* stream);
 
+/* The active-block list for callers that cannot allocate (the paper has no counterpart: this is
+ * about how the library is embedded, not about the method).  Some users of this library may not
+ * call cudaMalloc, or any allocator, at the point where the mask is rebuilt: code that runs as a
+ * plugin inside another framework's memory pool, a server that hands out all device memory at
+ * start-up, a latency-critical thread that must stay out of the allocator's lock.  Such a caller
+ * needs row_ptr / col_idx / tile_pairs for tra_sparse_attn and has no use for the Boolean mask, which
+ * is then scratch; this call keeps that scratch in a fixed array of TRA_STATIC_BLOCK_MASK_BYTES
+ * (16 MiB) inside the library's device image.  Every GPU on which the library is loaded holds those
+ * 16 MiB until the process exits.
+ *   Arguments and results as tra_build_block_mask without `block_mask`: the same row_ptr, col_idx,
+ *   nnz_out and tile_pairs, bit for bit; the same recorded errors.
+ *   Limit: B * heads * NB * NB <= TRA_STATIC_BLOCK_MASK_BYTES, else TRA_ERR_CAPACITY is returned and
+ *   nothing runs (the 75.6K-token, 40-head shape with 128-token blocks needs 13.97 MB).
+ *   The call itself allocates nothing: no cudaMalloc / cudaFree and no allocating library routine.
+ *   The first call on a device looks up the array's device address (once per device, with that device
+ *   current); make that first call before starting any stream capture.
+ *   All calls on a device share the one array, which keeps the last call's mask: two calls whose
+ *   kernels can overlap on the GPU (different streams without an ordering between them) race; order
+ *   them.  Nothing needs clearing between calls: a call writes every mask entry it later reads.
+ * Errors: TRA_ERR_INVALID_ARG (NULL pointer, non-positive count, a current device other than the
+ * plan's), TRA_ERR_CAPACITY (mask larger than the array, see above; or, recorded in the plan status,
+ * col_idx too small), TRA_ERR_UNSUPPORTED / TRA_ERR_CUDA as for tra_build_block_mask. */
+#define TRA_STATIC_BLOCK_MASK_BYTES (16u << 20)
+int tra_build_block_list_static(const tra_plan_t* plan, const uint16_t* ridx, int32_t* row_ptr,
+                                int32_t* col_idx, int64_t col_idx_capacity, int64_t* nnz_out,
+                                int32_t* tile_pairs, int B, int heads, void* stream);
+
 /* Block-sparse attention (Eq. 16 as executed: Section 3.2, last paragraph, and "Limitations"):
  * softmax attention of each query over the valid keys of the retained key blocks of its block row.
  *   ridx == NULL: retained blocks are evaluated in full, no token mask inside them (what the

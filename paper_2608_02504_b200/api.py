@@ -29,6 +29,7 @@ EXPORTS = [
     "tra_plan_num_radii", "tra_plan_tables", "tra_plan_count_table", "tra_plan_status",
     "tra_status_string", "tra_selftest_wait_timeout", "tra_tile_major_gather", "tra_tile_major_scatter",
     "tra_entropy_attn", "tra_budget_radius", "tra_build_block_mask", "tra_sparse_attn",
+    "tra_build_block_list_static",
     "tra_hot_path_host_workspace_bytes", "tra_hot_path_host",
 ]
 
@@ -71,6 +72,7 @@ def _load():
     lib.tra_budget_radius.argtypes = [vp, vp, vp, vp, vp, i32, i32, vp]
     lib.tra_build_block_mask.argtypes = [vp, vp, vp, vp, vp, ctypes.c_int64, vp, vp, i32, i32, vp]
     lib.tra_sparse_attn.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, vp]
+    lib.tra_build_block_list_static.argtypes = [vp, vp, vp, vp, ctypes.c_int64, vp, vp, i32, i32, vp]
     return lib
 
 
@@ -269,6 +271,20 @@ class Plan:
         if tile_pairs is not None:
             return block_mask, row_ptr, col_idx, nnz, tile_pairs
         return block_mask, row_ptr, col_idx, nnz
+
+    def build_block_list_static(self, ridx, row_ptr, col_idx, nnz=None, tile_pairs=None):
+        """ridx [B, heads, N] -> the active-block list, written into the caller's ``row_ptr`` / ``col_idx``
+        (and ``nnz`` / ``tile_pairs`` when given), through ``tra_build_block_list_static``: the variant of
+        ``build_block_mask`` for callers that must not allocate.  The Boolean mask stays in a fixed
+        16 MiB array inside the library, so every output must be passed in and nothing is created here;
+        shapes whose mask is larger raise ``TraError`` (TRA_ERR_CAPACITY)."""
+        B, heads = ridx.shape[0], ridx.shape[1]
+        _check(_lib.tra_build_block_list_static(self._h, _dev(ridx, torch.int16, "ridx"),
+                                                _dev(row_ptr, torch.int32, "row_ptr"),
+                                                _dev(col_idx, torch.int32, "col_idx"), col_idx.numel(),
+                                                _dev(nnz, torch.int64, "nnz"),
+                                                _dev(tile_pairs, torch.int32, "tile_pairs"), B, heads, _stream()),
+               "tra_build_block_list_static")
 
     def sparse_attn(self, Q, K, V, row_ptr, col_idx, O=None, lse=None, want_lse=False, sm_scale=None,
                     ridx=None, tile_pairs=None):

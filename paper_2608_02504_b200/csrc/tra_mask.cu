@@ -1,5 +1,6 @@
 // Block-mask construction from per-query radii (Algorithm 1) and its CSR active-block list.
 #include <algorithm>
+#include <mutex>
 
 #include "tra_common.cuh"
 
@@ -598,4 +599,52 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
     TRA_CUDA_CHECK(cudaGetLastError());
   }
   return TRA_OK;
+}
+
+
+// ---------------------------------------------------------------------------------------
+// Active-block list without any allocation.  A caller that only feeds tra_sparse_attn needs
+// row_ptr / col_idx (and the tile pairs); the Boolean mask between the vote and the list is then
+// scratch.  Here that scratch is a fixed array in the library's device image, so the call works
+// for code that may not allocate: a plugin running inside another framework's memory pool, a
+// serving loop whose device memory is fully committed at start-up, a real-time thread that must
+// not enter the allocator's lock.
+//
+// In host code `tra_static_block_mask` is only a handle of the symbol, not a device address; the
+// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that device
+// current, and is kept in g_static_mask_addr.
+// ---------------------------------------------------------------------------------------
+static __device__ __align__(256) uint8_t tra_static_block_mask[TRA_STATIC_BLOCK_MASK_BYTES];
+
+#define TRA_STATIC_MAX_DEVICES 64
+static uint8_t* g_static_mask_addr[TRA_STATIC_MAX_DEVICES];   // NULL until the device's first call
+static std::mutex g_static_mask_lock;
+
+extern "C" int tra_build_block_list_static(const tra_plan_t* plan, const uint16_t* ridx, int32_t* row_ptr,
+                                           int32_t* col_idx, int64_t col_idx_capacity, int64_t* nnz_out,
+                                           int32_t* tile_pairs, int B, int heads, void* stream) {
+  if (!plan || !ridx || !row_ptr || !col_idx || B < 1 || heads < 1 || col_idx_capacity < 0)
+    return TRA_ERR_INVALID_ARG;
+  int dev = -1;
+  TRA_CUDA_CHECK(cudaGetDevice(&dev));
+  if (dev != plan->device || dev < 0 || dev >= TRA_STATIC_MAX_DEVICES) return TRA_ERR_INVALID_ARG;
+  // the Boolean mask of this call must fit the fixed array
+  const long long need = (long long)B * heads * plan->NB * (long long)plan->NB;
+  if (need > (long long)TRA_STATIC_BLOCK_MASK_BYTES) return TRA_ERR_CAPACITY;
+  uint8_t* mask = nullptr;
+  {
+    std::lock_guard<std::mutex> guard(g_static_mask_lock);
+    if (!g_static_mask_addr[dev]) {
+      void* addr = nullptr;
+      if (cudaGetSymbolAddress(&addr, tra_static_block_mask) != cudaSuccess || !addr) {
+        cudaGetLastError();
+        return TRA_ERR_CUDA;
+      }
+      g_static_mask_addr[dev] = (uint8_t*)addr;
+    }
+    mask = g_static_mask_addr[dev];
+  }
+  // The vote writes every entry of the mask rows it owns, so nothing has to be cleared first.
+  return tra_build_block_mask(plan, ridx, mask, row_ptr, col_idx, col_idx_capacity, nnz_out, tile_pairs, B, heads,
+                              stream);
 }
