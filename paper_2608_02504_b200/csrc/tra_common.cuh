@@ -44,10 +44,12 @@ struct tra_plan {
   uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)
   uint32_t* d_counts_coarse;      // [T*H*W][16] every eighth entry of a row (n_radii <= 128), else NULL
   tra_block_boxes_t* d_boxes;     // [NB]
-  uint16_t* d_field_pos;          // where the block vote writes the count of frame cell (y, x), as an index into
-                                  // the frame's positions in tile-major order (the order repeats frame by frame):
-                                  // field_quads = 1: [H][W/4] index / 4 of the cells (y, 4j .. 4j+3), which are four
-                                  // consecutive positions starting at a multiple of four; else [H][W] one per cell
+  uint16_t* d_field_pos;          // block vote: where frame cell (y, x) sits in the frame's tile-major order (the
+                                  // order repeats frame by frame).  field_quads = 0: [H][W] the position of every
+                                  // cell; 1: [H][W/4] position / 4 of the cells (y, 4j .. 4j+3), which are four
+                                  // consecutive positions starting at a multiple of four, inside one block; 2:
+                                  // [H][W/16] position / 16 of the cells (y, 16m .. 16m+15), sixteen consecutive
+                                  // positions starting at a multiple of sixteen, inside one block
   int field_quads;
   int* d_status;                  // device status word
   // copy streams and events of tra_hot_path_host, created on its first calls with this plan and kept

@@ -29,13 +29,15 @@
 //    the whole frame at once: a query's disk meets row y' in the x-interval of half-width
 //    floor(sqrt(theta - (y'-y_i)^2)), which adds +1 / -1 to a difference array in shared
 //    memory (rows y_i - dy and y_i + dy share the half-width; a disk that covers the whole frame
-//    is only counted once).  One thread per row then takes the running sum along the row and
-//    stores the counts as bytes in the frame's tile-major order, so that the keys of a block are
-//    consecutive bytes.  Every undecided key block then reads the counts of its own keys in that
-//    frame (c_j by definition), four per 32-bit word, and compares all four with the two
-//    thresholds at once (adding 127 - t to a byte sets its top bit iff the byte exceeds t).  When
-//    the query block lies in one frame t0 the frames t0 - k and t0 + k see the same thresholds,
-//    so one field serves both.
+//    is only counted once).  The running sum along a row then gives the counts.  When four
+//    cells of a row are four consecutive tile-major positions of one key block (the usual
+//    case), the same pass compares the four counts, one per byte of a word, with the two
+//    thresholds at once (adding 127 - t to a byte sets its top bit iff the byte exceeds t) and adds
+//    the reached and high columns to the counter word of the key block they belong to: two threads
+//    per row, one summing from the left end, one from the right.  Otherwise one thread per row
+//    stores the counts as bytes in the frame's tile-major order and every undecided key block
+//    reads the counts of its own keys back, four per word.  When the query block lies in one
+//    frame t0 the frames t0 - k and t0 + k see the same thresholds, so one field serves both.
 // The outcome equals the unpruned vote bit for bit.
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ int tra_isqrt_small(int n) {
@@ -46,14 +48,24 @@ __device__ __forceinline__ int tra_isqrt_small(int n) {
   return (int)r;
 }
 
-// kQuads: the plan's position table has one entry per four cells of a row (see tra_plan::d_field_pos).
-template <bool kQuads>
-__global__ void __launch_bounds__(TRA_MASK_THREADS)
+__device__ __forceinline__ tra_box_t tra_load_box(const tra_box_t* p) {
+  union { int4 v; tra_box_t b; } u;
+  u.v = __ldg(reinterpret_cast<const int4*>(p));
+  return u.b;
+}
+
+// kMode = plan->field_quads.  0: the plan's position table has one entry per cell; 1: one entry per four cells of
+// a row (see tra_plan::d_field_pos); 2: moreover sixteen cells of a row are sixteen consecutive positions of one block.
+// ten resident CTAs per SM: 48 registers per thread without spills (12 CTAs, 40 registers, measured no faster)
+#define TRA_VOTE_MIN_CTAS 10
+template <int kMode>
+__global__ void __launch_bounds__(TRA_MASK_THREADS, TRA_VOTE_MIN_CTAS)
 tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restrict__ coord_packed,
                       const int32_t* __restrict__ theta, const tra_block_boxes_t* __restrict__ boxes,
                       const uint16_t* __restrict__ field_pos, uint8_t* __restrict__ block_mask,
                       int32_t* __restrict__ row_ptr, int N, int S, int NB, int NBv, int b, int T, int H, int W,
                       int n_radii, int keep_diagonal, int* __restrict__ status) {
+  constexpr bool kQuads = kMode != 0;
   extern __shared__ int32_t s_dyn[];
   __shared__ tra_block_boxes_t s_ubox;
   __shared__ int s_rstar, s_count, s_whole[2];
@@ -64,18 +76,23 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   int32_t* s_theta_star = s_dyn;                                   // [T]
   int32_t* s_frame_ylo = s_dyn + Tp;                               // [T] rows of the frame that hold keys of an
   int32_t* s_frame_yhi = s_dyn + 2 * Tp;                           // [T] undecided key block (yhi < 0: none)
-  int32_t* s_diff = s_dyn + 3 * Tp;                                // [H][Wp]
-  uint32_t* s_cols = (uint32_t*)(s_diff + n_diff);                 // [NB] reached columns | high columns << 16 |
+  int32_t* s_diff = s_dyn + 3 * Tp;                                // [H][Wp] (at least 320 words with kQuads)
+  const int diff_words = kQuads ? max(n_diff, 320) : n_diff;
+  uint32_t* s_cols = (uint32_t*)(s_diff + diff_words);             // [NB] reached columns | high columns << 16 |
                                                                    // state << 30 (0 / 1 decided, 2 undecided)
   const int HW = H * W;
-  const int n_pos = kQuads ? HW / 4 : HW;                          // entries of the position table
-  uint32_t* s_cnt = (uint32_t*)(s_dyn + 3 * Tp + n_diff + (NB + 3) / 4 * 4);   // [max(H * W, 1280)] bytes (16-byte
-                                                                   // aligned): counts in tile-major order
-  uint16_t* s_pos = (uint16_t*)(s_cnt + (max(HW, 1280) + 15) / 16 * 4);   // [n_pos] the plan's position table
-  // the sort of the queries by candidate index is over before the first counts are written
-  int* s_rank_key = (int*)s_cnt;                                   // [128]
-  uint32_t* s_sorted = s_cnt + 128;         // [128] queries in descending candidate index: coord, and ...
-  uint16_t* s_sorted_r = (uint16_t*)(s_cnt + 256);                 // [128] ... their candidate index
+  // entries of the plan's position table: per cell, per four cells, per sixteen cells
+  const int n_pos = kMode == 2 ? HW / 16 : (kQuads ? HW / 4 : HW);
+  const int cnt_bytes = kQuads ? 0 : max(HW, 1280);
+  uint32_t* s_cnt = s_cols + (NB + 3) / 4 * 4;                     // [cnt_bytes] bytes (16-byte aligned), without
+                                                                   // kQuads only: counts in tile-major order
+  uint16_t* s_pos = (uint16_t*)(s_cnt + (cnt_bytes + 15) / 16 * 4);       // [n_pos] the plan's position table
+  // The sort of the queries by candidate index borrows 1280 bytes: of the byte array (it is over before the first
+  // counts are written) or, with kQuads, of the count field (which is zeroed after the sort).
+  uint32_t* s_scratch = kQuads ? (uint32_t*)s_diff : s_cnt;
+  int* s_rank_key = (int*)s_scratch;                               // [128]
+  uint32_t* s_sorted = s_scratch + 128;     // [128] queries in descending candidate index: coord, and ...
+  uint16_t* s_sorted_r = (uint16_t*)(s_scratch + 256);             // [128] ... their candidate index
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int u = blockIdx.x;
@@ -115,8 +132,6 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     s_rstar = -1;
     s_whole[0] = s_whole[1] = 0;
   }
-  for (int i = tid; i < n_diff / 4; i += TRA_MASK_THREADS)   // the prefix pass leaves the rows it read zeroed again
-    reinterpret_cast<uint4*>(s_diff)[i] = make_uint4(0u, 0u, 0u, 0u);
   for (int i = tid; i < T; i += TRA_MASK_THREADS) {
     s_frame_ylo[i] = H;
     s_frame_yhi[i] = -1;
@@ -154,20 +169,29 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   __syncthreads();
 
   // ---- 1. classify every key block with the boxes -----------------------------------------
+  // (the count field starts all zero; every pass over its rows leaves them zeroed again)
+  for (int i = tid; i < n_diff / 4; i += TRA_MASK_THREADS)
+    reinterpret_cast<uint4*>(s_diff)[i] = make_uint4(0u, 0u, 0u, 0u);
   int kept = 0;
   for (int v = tid; v < NB; v += TRA_MASK_THREADS) {
     int decided = 0;   // 0 = vote 0, 1 = vote 1, 2 = undecided
-    tra_block_boxes_t vb;
-    vb.n_box = 0;
+    // the boxes of v sit in registers: five independent 16-byte loads, and loops over them that are unrolled in
+    // full (a private copy indexed by a loop variable would live in local memory)
+    tra_box_t vbox[TRA_MAX_SEG];
+    int vb_n = 0;
     if (v >= NBv) {
       decided = 1;     // text key block
     } else if (rstar >= 0) {
-      vb = boxes[v];
+#pragma unroll
+      for (int iv = 0; iv < TRA_MAX_SEG; ++iv) vbox[iv] = tra_load_box(boxes[v].box + iv);
+      vb_n = min(__ldg(&boxes[v].n_box), TRA_MAX_SEG);
       bool all_reject = true, all_accept = true;
       for (int iu = 0; iu < s_ubox.n_box; ++iu) {
         const tra_box_t a = s_ubox.box[iu];
-        for (int iv = 0; iv < vb.n_box; ++iv) {
-          const tra_box_t c = vb.box[iv];
+#pragma unroll
+        for (int iv = 0; iv < TRA_MAX_SEG; ++iv) {
+          if (iv >= vb_n) break;
+          const tra_box_t c = vbox[iv];
           int dt_min = max(0, max(a.t0 - c.t1, c.t0 - a.t1));
           int dt_max = max(a.t1 - c.t0, c.t1 - a.t0);
           int gy = max(0, max(a.y0 - c.y1, c.y0 - a.y1));
@@ -186,12 +210,16 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     s_cols[v] = (uint32_t)decided << 30;
     if (decided == 2) {
       // frames this key block has tokens in, and the rows of each that hold them
-      for (int iv = 0; iv < vb.n_box; ++iv)
-        for (int f = vb.box[iv].t0; f <= vb.box[iv].t1; ++f) {
+#pragma unroll
+      for (int iv = 0; iv < TRA_MAX_SEG; ++iv) {
+        if (iv >= vb_n) break;
+        const tra_box_t c = vbox[iv];
+        for (int f = c.t0; f <= c.t1; ++f) {
           if (!TRA_IDX(f, T, status)) break;
-          atomicMin(&s_frame_ylo[f], (int)vb.box[iv].y0);
-          atomicMax(&s_frame_yhi[f], (int)vb.box[iv].y1);
+          atomicMin(&s_frame_ylo[f], (int)c.y0);
+          atomicMax(&s_frame_yhi[f], (int)c.y1);
         }
+      }
     } else {
       mask_row[v] = (uint8_t)decided;
       kept += decided;
@@ -205,11 +233,14 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
   // number of queries whose disk covers the whole frame (they are left out of the field).
   // Only the rows win_lo .. win_hi of the frame are read afterwards: the field is built for them alone.
   int n_field = 0;
-  auto build_field = [&](auto dist_of_query, int win_lo, int win_hi) {
+  // Row intervals of every query's disk at the frame distance dist_of_query(), added to the difference array
+  // (rows win_lo .. win_hi only).  Ends with a barrier; returns the word that holds the number of queries whose
+  // disk covers the whole frame (they are left out of the field).
+  auto add_disk_rows = [&](auto dist_of_query, int win_lo, int win_hi) -> int* {
     // The field is all zero here (set at the start, and again by every prefix pass), and no warp still
-    // reads it: warps that lag behind are counting, which reads the byte array only.
+    // reads it.
     const int th = tid < nq ? __ldg(theta + qr * T + dist_of_query()) : 0;
-    int* whole = &s_whole[n_field & 1];     // alternates: the last field's readers may still be counting
+    int* whole = &s_whole[n_field & 1];     // alternates: the last field's readers may still be at work
     int* whole_next = &s_whole[++n_field & 1];
     if (tid < nq) {
       const int far_x = max(qx, W - 1 - qx), far_y = max(qy, H - 1 - qy);
@@ -222,6 +253,7 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
         const int d_first = max(0, max(win_lo - qy, qy - win_hi));
         const int d_last = min(R, max(qy - win_lo, win_hi - qy));
         const unsigned span = (unsigned)(win_hi - win_lo);
+#pragma unroll 2
         for (int dy = d_first; dy <= d_last; ++dy) {
           const int w = tra_isqrt_small(th - dy * dy);
           const int lo = max(0, qx - w), hi = min(W - 1, qx + w) + 1;      // lo < hi <= W < Wp
@@ -239,40 +271,103 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
     }
     __syncthreads();
     if (tid == 0) *whole_next = 0;          // its last readers passed the barrier above
-    // running sum along x, one thread per row; the counts (at most b <= 128) go out as bytes in tile-major
-    // order, and the row (column W included) is zeroed for the next field
-    for (int yy = win_lo + tid; yy <= win_hi; yy += TRA_MASK_THREADS) {
-      uint32_t run = 0;
-      if constexpr (kQuads) {
-        uint4* row = reinterpret_cast<uint4*>(s_diff + yy * Wp);
-        const uint16_t* pos = s_pos + yy * (W / 4);
-#pragma unroll 4
-        for (int j = 0; j < W / 4; ++j) {
+    return whole;
+  };
+  // A count c (without the `whole` queries) is reached iff c > -whole and high iff c > floor(b/3) - whole; with
+  // t >= -1 the byte c + (127 - t) <= 255 has its top bit set iff c > t (c <= b - whole, and t = -1 only when
+  // whole >= 1): four keys per 32-bit word are compared at once.
+  //
+  // Position table with one entry per four cells (kQuads): running sums and counting in one pass.  The row's
+  // differences sum to zero (every interval closes inside the row, column W included), so the count of a cell is
+  // the sum of the differences at and left of it, and also minus the sum of those right of it: the left half of
+  // a row is summed from the left by one thread (warps 0 and 1) and the right half from the right by another
+  // (warps 2 and 3).  Four cells of a row are four consecutive tile-major positions inside one key block (the
+  // block size is a multiple of four); their reached and high columns are added to the block's counter word
+  // whenever the block changes along the row.  fa / fb: the frames this field stands for (-1: not needed); the
+  // rows are zeroed again for the next field.  Ends with a barrier.
+  auto sum_and_count_rows = [&](int win_lo, int win_hi, int fa, int fb, int whole) {
+    const uint32_t add_reached = 0x01010101u * (uint32_t)(127 - max(-whole, -1));
+    const uint32_t add_high = 0x01010101u * (uint32_t)(127 - max(b / 3 - whole, -1));
+    const uint32_t magic = 0xffffffffu / (uint32_t)b + 1u;          // umulhi(p, magic) = p / b for p < 2^32 / b
+    const int nQ = W / 4, nL = (nQ + 1) / 2;                        // quads of a row; the left half's share
+    const bool right = tid >= TRA_MASK_THREADS / 2;
+    const uint32_t base_a = (uint32_t)((fa >= 0 ? fa : fb) * HW), base_b = (uint32_t)((fb >= 0 ? fb : fa) * HW);
+    for (int yy = win_lo + (tid & (TRA_MASK_THREADS / 2 - 1)); yy <= win_hi; yy += TRA_MASK_THREADS / 2) {
+      uint4* row = reinterpret_cast<uint4*>(s_diff + yy * Wp);
+      const uint16_t* pos = s_pos + yy * (kMode == 2 ? W / 16 : nQ);
+      uint32_t acc_r = 0, acc_h = 0, cur_a = 0xffffffffu, cur_b = 0xffffffffu;
+      auto flush = [&]() {
+        const uint32_t acc = acc_r + (acc_h << 16);
+        if (acc == 0) return;
+        if (fa >= 0 && TRA_IDX(cur_a, NB, status)) atomicAdd(&s_cols[cur_a], acc);
+        if (fb >= 0 && TRA_IDX(cur_b, NB, status)) atomicAdd(&s_cols[cur_b], acc);
+      };
+      // x: the counts of the quad's four cells, one per byte.  Its key block is looked up when it can differ from
+      // the previous quad's: for every quad, or (kMode 2) for the first quad met of every group of four.
+      auto count_quad = [&](int j, bool may_change, uint32_t x) {
+        if (may_change) {
+          const uint32_t p4 = kMode == 2 ? 16u * pos[j >> 2] : 4u * pos[j];
+          const uint32_t va = __umulhi(base_a + p4, magic), vb = __umulhi(base_b + p4, magic);
+          if (va != cur_a || vb != cur_b) {
+            flush();
+            acc_r = acc_h = 0;
+            cur_a = va;
+            cur_b = vb;
+          }
+        }
+        acc_r += __popc((x + add_reached) & 0x80808080u);
+        acc_h += __popc((x + add_high) & 0x80808080u);
+      };
+      // The packed counts come from multiplications: with differences d0..d3 and the count `run` left of the quad,
+      // run * 0x01010101 + d0 * 0x01010101 + d1 * 0x01010100 + d2 * 0x01010000 + d3 * 0x01000000 holds
+      // run + d0 + .. + dk in byte k (every such sum is a count in 0..128, so no byte borrows from its neighbour
+      // in the end, whatever the order of the additions modulo 2^32).  From the right: c3 = run, c2 = c3 - d3, ...
+      if (!right) {
+        uint32_t run = 0;
+#pragma unroll 1
+        for (int j = 0; j < nL; ++j) {
           const uint4 v = row[j];
           row[j] = make_uint4(0u, 0u, 0u, 0u);
-          const uint32_t c0 = run + v.x, c1 = c0 + v.y, c2 = c1 + v.z, c3 = c2 + v.w;
-          run = c3;
-          if (TRA_IDX(pos[j], HW / 4, status)) s_cnt[pos[j]] = c0 | (c1 << 8) | (c2 << 16) | (c3 << 24);
+          const uint32_t x = run * 0x01010101u + v.x * 0x01010101u + v.y * 0x01010100u + v.z * 0x01010000u +
+                             v.w * 0x01000000u;
+          run = x >> 24;
+          count_quad(j, kMode != 2 || (j & 3) == 0, x);
         }
-        row[W / 4] = make_uint4(0u, 0u, 0u, 0u);
       } else {
-        int32_t* row = s_diff + yy * Wp;
-        const uint16_t* pos = s_pos + yy * W;
-        for (int x = 0; x < W; ++x) {
-          run += (uint32_t)row[x];
-          row[x] = 0;
-          if (TRA_IDX(pos[x], HW, status)) reinterpret_cast<uint8_t*>(s_cnt)[pos[x]] = (uint8_t)run;
+        uint32_t run = 0u - row[nQ].x;                              // column W: minus the differences right of W - 1
+        row[nQ] = make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll 1
+        for (int j = nQ - 1; j >= nL; --j) {
+          const uint4 v = row[j];
+          row[j] = make_uint4(0u, 0u, 0u, 0u);
+          const uint32_t x = run * 0x01010101u - v.w * 0x00010101u - v.z * 0x00000101u - v.y;
+          run = (x & 0xffu) - v.x;
+          count_quad(j, kMode != 2 || (j & 3) == 3 || j == nQ - 1, x);
         }
-        row[W] = 0;
       }
+      flush();
     }
     __syncthreads();
-    return *whole;
   };
-  // undecided key blocks with tokens in frame f read their keys' counts: one warp per block, four keys
-  // per lane and word.  A count c (without the `whole` queries) is reached iff c > -whole and high iff
-  // c > floor(b/3) - whole; with t >= -1 the byte c + (127 - t) <= 255 has its top bit set iff c > t
-  // (c <= b - whole, and t = -1 only when whole >= 1).
+  // Position table with one entry per cell: running sum along x, one thread per row; the counts (at most
+  // b <= 128) go out as bytes in tile-major order, and the row (column W included) is zeroed for the next field.
+  // Ends with a barrier.
+  auto sum_rows_to_bytes = [&](int win_lo, int win_hi) {
+    for (int yy = win_lo + tid; yy <= win_hi; yy += TRA_MASK_THREADS) {
+      uint32_t run = 0;
+      int32_t* row = s_diff + yy * Wp;
+      const uint16_t* pos = s_pos + yy * W;
+      for (int x = 0; x < W; ++x) {
+        run += (uint32_t)row[x];
+        row[x] = 0;
+        if (TRA_IDX(pos[x], HW, status)) reinterpret_cast<uint8_t*>(s_cnt)[pos[x]] = (uint8_t)run;
+      }
+      row[W] = 0;
+    }
+    __syncthreads();
+  };
+  // ... after which the undecided key blocks with tokens in frame f read their keys' counts: one warp per block,
+  // four keys per lane and word.
   auto count_frame = [&](int f, int whole) {
     const uint32_t add_reached = 0x01010101u * (uint32_t)(127 - max(-whole, -1));
     const uint32_t add_high = 0x01010101u * (uint32_t)(127 - max(b / 3 - whole, -1));
@@ -298,6 +393,17 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       if (lane == 0) s_cols[v] += (uint32_t)acc;   // one warp owns v inside a frame; frames are processed in turn
     }
   };
+  // the field of one frame distance, counted for the frames fa and fb (-1: not needed)
+  auto field = [&](auto dist_of_query, int win_lo, int win_hi, int fa, int fb) {
+    const int whole = *add_disk_rows(dist_of_query, win_lo, win_hi);
+    if constexpr (kQuads) {
+      sum_and_count_rows(win_lo, win_hi, fa, fb, whole);
+    } else {
+      sum_rows_to_bytes(win_lo, win_hi);
+      if (fa >= 0) count_frame(fa, whole);
+      if (fb >= 0) count_frame(fb, whole);
+    }
+  };
   // A query block that lies in one frame t0 sees frames t0 - k and t0 + k at the same distance:
   // their fields are the same, so one field serves both.
   bool one_frame = s_ubox.n_box > 0;
@@ -313,15 +419,12 @@ tra_block_vote_kernel(const uint16_t* __restrict__ ridx, const uint32_t* __restr
       int win_lo = min(need_a ? s_frame_ylo[fa] : H, need_b ? s_frame_ylo[fb] : H);
       int win_hi = max(need_a ? s_frame_yhi[fa] : -1, need_b ? s_frame_yhi[fb] : -1);
       if (!TRA_IDX(win_lo, H, status) || !TRA_IDX(win_hi, H, status)) win_lo = 0, win_hi = H - 1;
-      const int whole = build_field([&]() { return k; }, win_lo, win_hi);
-      if (need_a) count_frame(fa, whole);
-      if (need_b) count_frame(fb, whole);
+      field([&]() { return k; }, win_lo, win_hi, need_a ? fa : -1, need_b ? fb : -1);
     }
   } else {
     for (int f = 0; f < T; ++f) {
       if (s_frame_yhi[f] < 0) continue;                 // uniform across the CTA
-      const int whole = build_field([&]() { return abs(qt - f); }, s_frame_ylo[f], s_frame_yhi[f]);
-      count_frame(f, whole);
+      field([&]() { return abs(qt - f); }, s_frame_ylo[f], s_frame_yhi[f], f, -1);
     }
   }
 
@@ -559,12 +662,18 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   const long long rows = BH * NB;
 
   const int H = plan->cfg.H, W = plan->cfg.W;
-  size_t smem = ((size_t)3 * ((T + 3) & ~3) + (size_t)H * tra_field_row_words(W)) * sizeof(int32_t) +
-                ((size_t)NB + 3) / 4 * 16 + (std::max<size_t>((size_t)H * W, 1280) + 15) / 16 * 16 +
-                ((((size_t)H * W / (plan->field_quads ? 4 : 1)) + 7) & ~(size_t)7) * sizeof(uint16_t);
+  // thresholds and frame windows, count field, counter words, byte array (without quads), position table:
+  // the layout at the top of the kernel
+  const int mode = plan->field_quads;
+  const size_t n_diff = (size_t)H * tra_field_row_words(W);
+  const size_t n_pos = (size_t)H * W / (mode == 2 ? 16 : (mode ? 4 : 1));
+  size_t smem = ((size_t)3 * ((T + 3) & ~3) + (mode ? std::max<size_t>(n_diff, 320) : n_diff)) * sizeof(int32_t) +
+                ((size_t)NB + 3) / 4 * 16 + (mode ? 0 : (std::max<size_t>((size_t)H * W, 1280) + 15) / 16 * 16) +
+                ((n_pos + 7) & ~(size_t)7) * sizeof(uint16_t);
   if (smem > 200 * 1024 || !plan->d_field_pos) return TRA_ERR_UNSUPPORTED;   // frame too large for the count field
   dim3 grid((unsigned)NB, (unsigned)BH);
-  auto vote = plan->field_quads ? tra_block_vote_kernel<true> : tra_block_vote_kernel<false>;
+  auto vote = plan->field_quads == 2 ? tra_block_vote_kernel<2>
+                                     : (plan->field_quads ? tra_block_vote_kernel<1> : tra_block_vote_kernel<0>);
   if (smem > 48 * 1024)
     TRA_CUDA_CHECK(cudaFuncSetAttribute(vote, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   vote<<<grid, TRA_MASK_THREADS, smem, stream>>>(

@@ -277,14 +277,20 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   if (field_pos_fits) {
     std::vector<int32_t> pos_of((size_t)H * W);
     for (int i = 0; i < H * W; ++i) pos_of[(size_t)p->h_coord[3 * i + 1] * W + p->h_coord[3 * i + 2]] = i;
-    bool quads = W % 4 == 0;
+    bool quads = W % 4 == 0 && cfg->block % 4 == 0;      // a group of four positions never straddles two blocks
     for (int c = 0; c < H * W && quads; c += 4)
       quads = pos_of[c] % 4 == 0 && pos_of[c + 1] == pos_of[c] + 1 && pos_of[c + 2] == pos_of[c] + 2 &&
               pos_of[c + 3] == pos_of[c] + 3;
-    p->field_quads = quads ? 1 : 0;
-    const size_t n = quads ? (size_t)H * W / 4 : (size_t)H * W;
+    // 2: moreover the sixteen cells (y, 16 m .. 16 m + 15) are sixteen consecutive positions that start at a
+    // multiple of sixteen and lie inside one block in every frame
+    bool seg16 = quads && W % 16 == 0 && cfg->block % 16 == 0;
+    for (int c = 0; c < H * W && seg16; c += 16)
+      for (int i = 0; i < 16 && seg16; ++i) seg16 = pos_of[c] % 16 == 0 && pos_of[c + i] == pos_of[c] + i;
+    p->field_quads = seg16 ? 2 : (quads ? 1 : 0);
+    const int per = seg16 ? 16 : (quads ? 4 : 1);        // cells per entry: entry i = position of cell i * per, / per
+    const size_t n = (size_t)H * W / per;
     field_pos.assign((n + 7) & ~(size_t)7, 0);
-    for (size_t i = 0; i < n; ++i) field_pos[i] = (uint16_t)(quads ? pos_of[4 * i] / 4 : pos_of[i]);
+    for (size_t i = 0; i < n; ++i) field_pos[i] = (uint16_t)(pos_of[per * i] / per);
   }
 
   // device tables
