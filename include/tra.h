@@ -166,7 +166,11 @@ int tra_budget_radius(const tra_plan_t* plan, const float* entropy, int32_t* bud
  *               lists are similar (entry -1 = no second tile).  Pass it to tra_sparse_attn together
  *               with row_ptr / col_idx; it changes the speed of that call, never its result.
  *               Block sizes that do not divide 128 have no attention launch and no query tiles:
- *               with such a plan a non-NULL tile_pairs returns TRA_ERR_UNSUPPORTED (nothing is run). */
+ *               with such a plan a non-NULL tile_pairs returns TRA_ERR_UNSUPPORTED (nothing is run).
+ *               The pairing kernel runs beside the list kernels on a stream the plan owns, forked from and
+ *               joined to `stream` by two plan-owned events (this also works inside a stream capture):
+ *               everything the call writes is complete for later work on `stream`, but calls with
+ *               tile_pairs on ONE plan must not be issued from several host threads at once. */
 int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx, uint8_t* block_mask,
                          int32_t* row_ptr, int32_t* col_idx, int64_t col_idx_capacity,
                          int64_t* nnz_out, int32_t* tile_pairs, int B, int heads, void* stream);

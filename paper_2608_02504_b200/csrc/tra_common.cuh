@@ -42,7 +42,8 @@ struct tra_plan {
   int32_t* d_theta;               // [n_radii][T]
   float* d_radii_f32;             // [n_radii]
   uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)
-  uint32_t* d_counts_coarse;      // [T*H*W][16] every eighth entry of a row (n_radii <= 128), else NULL
+  uint32_t* d_counts_coarse;      // n_radii <= 128: [T*H*W][16] every eighth entry of a row, then [T*H*W][128] the
+                                  // rows padded to 128 entries (sector-aligned groups of eight); else NULL
   tra_block_boxes_t* d_boxes;     // [NB]
   uint16_t* d_field_pos;          // block vote: where frame cell (y, x) sits in the frame's tile-major order (the
                                   // order repeats frame by frame).  field_quads = 0: [H][W] the position of every
@@ -52,6 +53,10 @@ struct tra_plan {
                                   // positions starting at a multiple of sixteen, inside one block
   int field_quads;
   int* d_status;                  // device status word
+  // tra_build_block_mask: the tile-pair kernel runs on a stream of its own beside the list kernels (fork and join
+  // events on the caller's stream); created with the plan
+  cudaStream_t pair_stream;
+  cudaEvent_t pair_fork, pair_join;
   // copy streams and events of tra_hot_path_host, created on its first calls with this plan and kept
   cudaStream_t copy_in, copy_out;
   cudaEvent_t* events;

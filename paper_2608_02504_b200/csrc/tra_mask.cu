@@ -671,6 +671,24 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
                 ((size_t)NB + 3) / 4 * 16 + (mode ? 0 : (std::max<size_t>((size_t)H * W, 1280) + 15) / 16 * 16) +
                 ((n_pos + 7) & ~(size_t)7) * sizeof(uint16_t);
   if (smem > 200 * 1024 || !plan->d_field_pos) return TRA_ERR_UNSUPPORTED;   // frame too large for the count field
+  // tile pairing (checked before anything is launched)
+  int G = 1, NT = 0, frame_tiles = 0;
+  size_t pair_smem = 0;
+  if (tile_pairs) {
+    // query tiles of the attention launch: 128 rows = G blocks
+    const int b = plan->cfg.block;
+    G = 128 / b;
+    NT = (NB + G - 1) / G;
+    // tiles per frame, rounded: the tile one frame ahead of u is u + frame_tiles or a neighbour of it
+    const long long tile_tokens = (long long)b * G;
+    frame_tiles = (int)(((long long)plan->cfg.H * plan->cfg.W + tile_tokens / 2) / tile_tokens);
+    const int reach = frame_tiles - 1 > TRA_PAIR_WINDOW ? frame_tiles + 1 : TRA_PAIR_WINDOW;
+    pair_smem = ((size_t)(TRA_PAIR_CHUNK + reach) * ((NB + 31) / 32)) * 4 + (size_t)NT * TRA_PAIR_CANDS * 2;
+    if (pair_smem > 200 * 1024 || NT > 2048) return TRA_ERR_UNSUPPORTED;
+    if (pair_smem > 48 * 1024)
+      TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)pair_smem));
+  }
   dim3 grid((unsigned)NB, (unsigned)BH);
   auto vote = plan->field_quads == 2 ? tra_block_vote_kernel<2>
                                      : (plan->field_quads ? tra_block_vote_kernel<1> : tra_block_vote_kernel<0>);
@@ -681,32 +699,24 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
       plan->S, NB, plan->NBv, plan->cfg.block, T, H, W, plan->n_radii, (plan->cfg.flags & TRA_KEEP_DIAGONAL) ? 1 : 0,
       plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
+  // The tile pairs need the Boolean mask only, the list kernels too: the pairing runs beside them on the plan's
+  // own stream, forked from and joined to the caller's stream by events (legal inside a stream capture as well).
+  if (tile_pairs) {
+    const unsigned n_seg = (unsigned)std::max(1ll, std::min(4ll, (long long)plan->sm_count / BH));   // one CTA per SM
+    TRA_CUDA_CHECK(cudaEventRecord(plan->pair_fork, stream));
+    TRA_CUDA_CHECK(cudaStreamWaitEvent(plan->pair_stream, plan->pair_fork, 0));
+    tra_pair_tiles_kernel<<<dim3((unsigned)BH, n_seg), TRA_PAIR_THREADS, pair_smem, plan->pair_stream>>>(
+        block_mask, tile_pairs, NB, NT, G, frame_tiles, plan->d_status);
+    TRA_CUDA_CHECK(cudaGetLastError());
+    TRA_CUDA_CHECK(cudaEventRecord(plan->pair_join, plan->pair_stream));
+  }
   tra_row_ptr_scan_kernel<<<1, 1024, 0, stream>>>(row_ptr, rows, (long long)col_idx_capacity, nnz_out,
                                                   plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
   tra_col_idx_fill_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, stream>>>(
       block_mask, row_ptr, col_idx, rows, NB, (long long)col_idx_capacity, plan->d_status);
   TRA_CUDA_CHECK(cudaGetLastError());
-  if (tile_pairs) {
-    // query tiles of the attention launch: 128 rows = G blocks
-    const int b = plan->cfg.block;
-    const int G = 128 / b;
-    const int NT = (NB + G - 1) / G;
-    // tiles per frame, rounded: the tile one frame ahead of u is u + frame_tiles or a neighbour of it
-    const long long tile_tokens = (long long)b * G;
-    const int frame_tiles = (int)(((long long)plan->cfg.H * plan->cfg.W + tile_tokens / 2) / tile_tokens);
-    const int reach = frame_tiles - 1 > TRA_PAIR_WINDOW ? frame_tiles + 1 : TRA_PAIR_WINDOW;
-    const size_t pair_smem = ((size_t)(TRA_PAIR_CHUNK + reach) * ((NB + 31) / 32)) * 4 +
-                             (size_t)NT * TRA_PAIR_CANDS * 2;
-    if (pair_smem > 200 * 1024 || NT > 2048) return TRA_ERR_UNSUPPORTED;
-    if (pair_smem > 48 * 1024)
-      TRA_CUDA_CHECK(cudaFuncSetAttribute(tra_pair_tiles_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)pair_smem));
-    const unsigned n_seg = (unsigned)std::max(1ll, std::min(4ll, (long long)plan->sm_count / BH));   // one CTA per SM
-    tra_pair_tiles_kernel<<<dim3((unsigned)BH, n_seg), TRA_PAIR_THREADS, pair_smem, stream>>>(
-        block_mask, tile_pairs, NB, NT, G, frame_tiles, plan->d_status);
-    TRA_CUDA_CHECK(cudaGetLastError());
-  }
+  if (tile_pairs) TRA_CUDA_CHECK(cudaStreamWaitEvent(stream, plan->pair_join, 0));
   return TRA_OK;
 }
 

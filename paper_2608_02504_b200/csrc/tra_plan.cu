@@ -109,6 +109,9 @@ static void tra_plan_free(tra_plan* p) {
   cudaFree(p->d_boxes);
   cudaFree(p->d_field_pos);
   cudaFree(p->d_status);
+  if (p->pair_stream) cudaStreamDestroy(p->pair_stream);
+  if (p->pair_fork) cudaEventDestroy(p->pair_fork);
+  if (p->pair_join) cudaEventDestroy(p->pair_join);
   if (p->copy_in) cudaStreamDestroy(p->copy_in);
   if (p->copy_out) cudaStreamDestroy(p->copy_out);
   for (int i = 0; i < p->n_events; ++i) cudaEventDestroy(p->events[i]);
@@ -301,10 +304,13 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
             cudaMalloc(&p->d_theta, sizeof(int32_t) * nr * T) == cudaSuccess &&
             cudaMalloc(&p->d_radii_f32, sizeof(float) * nr) == cudaSuccess &&
             cudaMalloc(&p->d_counts, sizeof(uint32_t) * count_elems) == cudaSuccess &&
-            (nr > 128 || cudaMalloc(&p->d_counts_coarse, sizeof(uint32_t) * 16 * (size_t)p->N) == cudaSuccess) &&
+            (nr > 128 || cudaMalloc(&p->d_counts_coarse, sizeof(uint32_t) * (16 + 128) * (size_t)p->N) == cudaSuccess) &&
             cudaMalloc(&p->d_boxes, sizeof(tra_block_boxes_t) * p->NB) == cudaSuccess &&
             (!field_pos_fits || cudaMalloc(&p->d_field_pos, sizeof(uint16_t) * field_pos.size()) == cudaSuccess) &&
-            cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess;
+            cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p->pair_stream, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p->pair_fork, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&p->pair_join, cudaEventDisableTiming) == cudaSuccess;
   ok = ok &&
        cudaMemcpyAsync(p->d_coord_packed, packed.data(), sizeof(uint32_t) * (p->N + 128),
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&

@@ -46,7 +46,8 @@ __device__ __forceinline__ const uint32_t* tra_count_row(const RadiusArgs& a, ui
 // of independent loads instead of seven dependent ones.  Round 1 reads the token's row of the coarse
 // table (every eighth entry of its count-table row, 64 bytes, four 16-byte loads) and counts the
 // entries below the budget, which names the group of eight that holds the answer; round 2 reads
-// that group and counts again.  Rows are non-decreasing, so "entries below the budget" is the index
+// that group (one aligned 32-byte sector of a copy of the count table with rows padded to 128
+// entries; the rows of the table itself are not sector-aligned) and counts again.  Rows are non-decreasing, so "entries below the budget" is the index
 // of the first entry that reaches it (Eq. 14).
 __global__ void __launch_bounds__(256) tra_budget_radius_2round_kernel(RadiusArgs a, const uint32_t* __restrict__ coarse) {
   const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -67,29 +68,33 @@ __global__ void __launch_bounds__(256) tra_budget_radius_2round_kernel(RadiusArg
   const int grp = (q0.x < need) + (q0.y < need) + (q0.z < need) + (q0.w < need) + (q1.x < need) + (q1.y < need) +
                   (q1.z < need) + (q1.w < need) + (q2.x < need) + (q2.y < need) + (q2.z < need) + (q2.w < need) +
                   (q3.x < need) + (q3.y < need) + (q3.z < need) + (q3.w < need);
-  const uint32_t* row = a.counts + cell * a.n_radii;
-  const int base = grp * 8;            // grp <= (n_radii - 1) / 8: the last entry of a row is N >= need
-  uint32_t e[8];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) e[j] = base + j < a.n_radii ? __ldg(row + base + j) : 0xffffffffu;
-  int lo = base;
-#pragma unroll
-  for (int j = 0; j < 8; ++j) lo += e[j] < need;
+  // the group of eight: one aligned 32-byte sector of the padded copy of the count table that follows the
+  // coarse table (rows of 128 entries, the entries past n_radii hold the largest value)
+  const int base = min(grp, 15) * 8;   // grp <= (n_radii - 1) / 8: the last entry of a row is N >= need
+  const uint4* fr = reinterpret_cast<const uint4*>(coarse + (size_t)a.N * 16 + cell * 128 + base);
+  const uint4 e0 = __ldg(fr), e1 = __ldg(fr + 1);
+  int lo = base + (e0.x < need) + (e0.y < need) + (e0.z < need) + (e0.w < need) + (e1.x < need) + (e1.y < need) +
+           (e1.z < need) + (e1.w < need);
   if (!TRA_IDX(lo, a.n_radii, a.status)) lo = a.n_radii - 1;
   if (a.budget) a.budget[g] = (int32_t)need;
   if (a.radius) a.radius[g] = __ldg(a.radii + lo);
   a.ridx[g] = (uint16_t)lo;
 }
 
-// coarse[cell][i] = counts[cell][min(8 i + 7, n_radii - 1)] for the groups that exist, else the largest value.
+// coarse[cell][i] = counts[cell][min(8 i + 7, n_radii - 1)] for the groups that exist, else the largest value;
+// behind the coarse table, padded[cell][j] = counts[cell][j] for j < n_radii, else the largest value (j < 128).
 __global__ void tra_coarse_table_kernel(const uint32_t* __restrict__ counts, uint32_t* __restrict__ coarse,
                                         long long cells, int n_radii, int* __restrict__ status) {
   const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= cells * 16) return;
-  const long long cell = g >> 4;
-  const int i = (int)(g & 15);
-  const long long src = cell * n_radii + min(8 * i + 7, n_radii - 1);
-  coarse[g] = 8 * i < n_radii && TRA_IDX(src, cells * n_radii, status) ? counts[src] : 0xffffffffu;
+  if (g >= cells * 128) return;
+  const long long cell = g >> 7;
+  const int j = (int)(g & 127);
+  const long long src_j = cell * n_radii + j;
+  coarse[cells * 16 + g] = j < n_radii && TRA_IDX(src_j, cells * n_radii, status) ? counts[src_j] : 0xffffffffu;
+  if (j < 16) {
+    const long long src = cell * n_radii + min(8 * j + 7, n_radii - 1);
+    coarse[cell * 16 + j] = 8 * j < n_radii && TRA_IDX(src, cells * n_radii, status) ? counts[src] : 0xffffffffu;
+  }
 }
 
 // Binary search in the count-table row: candidate sets of more than 128 radii.
@@ -118,10 +123,11 @@ __global__ void __launch_bounds__(256) tra_budget_radius_kernel(RadiusArgs a) {
 
 }  // namespace
 
-// Plan time: the coarse table of the two-round search (called by tra_plan_create for sets of <= 128 radii).
+// Plan time: the coarse table of the two-round search and the padded copy of the count table behind it, 16 + 128
+// words per cell (called by tra_plan_create for sets of <= 128 radii).
 int tra_build_coarse_table(const uint32_t* counts, uint32_t* coarse, long long cells, int n_radii, int* status,
                            cudaStream_t stream) {
-  const long long total = cells * 16;
+  const long long total = cells * 128;
   tra_coarse_table_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(counts, coarse, cells, n_radii,
                                                                                status);
   return cudaGetLastError() == cudaSuccess ? TRA_OK : TRA_ERR_CUDA;
