@@ -167,6 +167,43 @@ def test_block_mask_bit_exact(cfg, kind):
         plan.close()
 
 
+# The vote kernel has three layouts of its per-frame count field, chosen by the plan: sixteen cells of a row are
+# one run of positions inside a block (W, tile width and block multiples of 16), four cells are (multiples of 4),
+# or neither.  Full-size shapes use the first; these small grids cover all three, with blocks that straddle tiles
+# and frames, a ragged last block, and text tokens.
+VOTE_LAYOUT_CASES = [
+    ("runs of 16, b=128", common.small_config(4, 12, 32, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16, seed=91)),
+    ("runs of 16, b=64", common.small_config(3, 8, 48, heads=2, head_dim=64, block=64, tile_h=4, tile_w=16, seed=92)),
+    ("runs of 16, b=48", common.small_config(3, 10, 32, heads=2, head_dim=128, block=48, tile_h=8, tile_w=16, seed=93)),
+    ("runs of 16, b=80, tile 2x32", common.small_config(5, 7, 32, heads=2, head_dim=128, block=80, tile_h=2, tile_w=32, seed=94)),
+    ("runs of 4, b=64", common.small_config(4, 9, 24, heads=2, head_dim=64, block=64, tile_h=4, tile_w=8, seed=95)),
+    ("runs of 4, b=36", common.small_config(3, 11, 20, heads=2, head_dim=128, block=36, tile_h=4, tile_w=4, seed=96)),
+    ("runs of 4 only (b=40)", common.small_config(3, 6, 32, heads=2, head_dim=128, block=40, tile_h=2, tile_w=16, seed=97)),
+    ("single cells (b=30)", common.small_config(3, 6, 32, heads=2, head_dim=128, block=30, tile_h=2, tile_w=16, seed=98)),
+    ("single cells (W=10)", common.small_config(4, 9, 10, heads=2, head_dim=64, block=64, tile_h=4, tile_w=4, seed=99)),
+]
+
+
+@pytest.mark.parametrize("name,cfg", VOTE_LAYOUT_CASES, ids=[c[0] for c in VOTE_LAYOUT_CASES])
+@pytest.mark.parametrize("n_text", [0, 45])
+def test_block_vote_count_field_layouts(name, cfg, n_text):
+    geo = common.oracle_geometry(cfg)
+    heads = cfg["heads"]
+    for kind, flags in (("entropy", 0), ("uniform", api().TRA_KEEP_DIAGONAL), ("small", 0), ("blocky", 0)):
+        ridx = random_ridx(geo, heads, np.random.default_rng(31), kind)
+        plan = make_plan(cfg, flags=flags, n_text=n_text)
+        S = geo.N + n_text
+        full = np.full((heads, S), geo.radii.size - 1, np.uint16)      # text positions: the last candidate
+        full[:, : geo.N] = ridx
+        mask, row_ptr, col_idx, nnz = run_mask(plan, full)
+        ref = np.stack([oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, full[h], keep_diagonal=bool(flags),
+                                          n_text=n_text) for h in range(heads)])
+        assert np.array_equal(mask, ref), (name, kind)
+        rp, ci = oracle.csr_from_block_mask(ref)
+        assert nnz == rp[-1] and np.array_equal(row_ptr.astype(np.int64), rp) and np.array_equal(col_idx[:nnz], ci)
+        plan.close()
+
+
 def _random_geometries(n, seed):
     rng = np.random.default_rng(seed)
     out = []
