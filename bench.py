@@ -67,9 +67,67 @@ def load_peaks():
     return p
 
 
+class NvmlSampler:
+    """Samples the SM clock and the clock-event reasons through NVML (read-only queries) every 50 ms from a
+    thread, between window() and stop().  nvidia-smi in loop mode delivers only about one line per second while
+    the GPU is busy, which leaves a three-second timed region with a handful of samples; ClockSampler below is
+    the fallback when the NVML binding is missing."""
+
+    def __init__(self, gpu_index):
+        import threading
+        import pynvml
+        self.nv = pynvml
+        pynvml.nvmlInit()
+        try:
+            uuid = str(torch.cuda.get_device_properties(gpu_index).uuid)
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+        except Exception:
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+        self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        self.samples, self.mask, self.on, self.done = [], 0, False, False
+        self.thread = threading.Thread(target=self._run, daemon=True)
+
+    def start(self):
+        self.thread.start()
+
+    def _run(self):
+        nv = self.nv
+        while not self.done:
+            if self.on:
+                try:
+                    self.samples.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                    self.mask |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    pass
+            time.sleep(0.05)
+
+    def window(self, t_begin, t_end):
+        self.on = t_end is None         # window(t, None) opens the sampling window, stop() closes it
+
+    def stop(self):
+        self.on, self.done = False, True
+        self.thread.join(timeout=2)
+        nv = self.nv
+        names = [("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
+                 ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                 ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
+                 ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap)]
+        reasons = sorted(n for n, bit in names if self.mask & bit)
+        busy = [c for c in self.samples if c > 0]
+        return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": self.smax, "reasons": reasons,
+                "samples": len(self.samples), "source": "nvml, every 50 ms"}
+
+
+def make_sampler(gpu_index):
+    try:
+        return NvmlSampler(gpu_index)
+    except Exception:
+        return ClockSampler(gpu_index)
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -87,6 +145,20 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def window(self, t_begin, t_end):
+        """Only samples taken between these two time.time() values count (the sampler is started well before
+        the timed region, because nvidia-smi takes a second or two to deliver its first line)."""
+        if t_end is not None:
+            self.t_begin, self.t_end = t_begin, t_end
+
+    @staticmethod
+    def _stamp(text):
+        import datetime
+        try:
+            return datetime.datetime.strptime(text, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -101,6 +173,10 @@ class ClockSampler:
             for line in open(self.path):
                 f = [x.strip() for x in line.split(",")]
                 if len(f) < 9:
+                    continue
+                ts = self._stamp(f[0])
+                if ts is not None and getattr(self, "t_begin", None) is not None and \
+                        not (self.t_begin <= ts <= self.t_end + 0.2):
                     continue
                 try:
                     sm.append(float(f[1]))
@@ -216,6 +292,8 @@ def run_ours(args):
     N, d, block = workloads.num_tokens(cfg), cfg["head_dim"], cfg["block"]
     peaks = load_peaks()
 
+    sampler = make_sampler(local)
+    sampler.start()                     # started early; only samples of the timed region count
     plan = api.Plan.from_config(cfg)
     Qr, Kr, Vr = workloads.make_qkv(cfg, dev, heads=my_heads)
     NB = plan.NB
@@ -277,16 +355,16 @@ def run_ours(args):
 
     # ---- timed region: K steps, device-timed, inputs resident in HBM -----------------------
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
-    sampler = ClockSampler(local)
     barrier(world)
     torch.cuda.synchronize()
-    sampler.start()
     t_wall = time.time()
+    sampler.window(t_wall, None)
     for k in range(args.steps):
         one_step(ev[k])
     torch.cuda.synchronize()
     barrier(world)
     wall_s = time.time() - t_wall
+    sampler.window(t_wall, t_wall + wall_s)
     clocks = sampler.stop()
     total_ms = reduce_over_ranks(ev[0][0].elapsed_time(ev[-1][6]), world, dev)
     plan.check_status()
