@@ -67,8 +67,9 @@ typedef struct tra_plan tra_plan_t; /* opaque: grid geometry, thresholds, count 
 typedef struct {
   int T, H, W;         /* latent grid (Section 2.1); 1 <= T,H,W <= 1023                          */
   int head_dim;        /* d: 64 or 128                                                          */
-  int block;           /* b of Algorithm 1: 64 or 128 for the attention calls; 16..128 for the   */
-                       /* budget/radius/mask calls                                              */
+  int block;           /* b of Algorithm 1: 16..128 for the budget/radius/mask calls; the        */
+                       /* attention calls take 33..128 with head_dim 128 (64 or 128 with        */
+                       /* head_dim 64); the token mask inside blocks (ridx) needs 64 or 128     */
   int tile_h, tile_w;  /* tile shape of the tile-major order (Section 3.3)                       */
   double tau;          /* target attention mass of Eq. 4, in (0, 1]                              */
   double gamma;        /* temporal decay rate of Eq. 10, >= 0                                    */
@@ -160,12 +161,14 @@ int tra_budget_radius(const tra_plan_t* plan, const float* entropy, int32_t* bud
  *               offset is clamped to the capacity, so that a later tra_sparse_attn stays inside
  *               col_idx (its result is then incomplete; read the status).
  *   nnz_out   : device int64 or NULL; total retained blocks.
- *   tile_pairs: int32 [B*heads, ceil(NT/2), 2] or NULL, NT = ceil(S / 128) (written).  The paper has
- *               no counterpart: tra_sparse_attn gives each thread block two 128-row query tiles that
+ *   tile_pairs: int32 [B*heads, ceil(NT/2), 2] or NULL, NT = ceil(NB / G) query tiles, G = 2 blocks
+ *               per tile for blocks of up to 64 tokens, else 1 (written).  The paper has
+ *               no counterpart: tra_sparse_attn gives each thread block two query tiles (128 rows of
+ *               tensor-core work each, of which the first G * block hold queries) that
  *               share the key/value tiles they both retain, and this table pairs tiles whose block
  *               lists are similar (entry -1 = no second tile).  Pass it to tra_sparse_attn together
  *               with row_ptr / col_idx; it changes the speed of that call, never its result.
- *               Block sizes that do not divide 128 have no attention launch and no query tiles:
+ *               Blocks of 32 tokens or fewer have no attention launch and no query tiles:
  *               with such a plan a non-NULL tile_pairs returns TRA_ERR_UNSUPPORTED (nothing is run).
  *               The pairing kernel runs beside the list kernels on a stream the plan owns, forked from and
  *               joined to `stream` by two plan-owned events (this also works inside a stream capture):

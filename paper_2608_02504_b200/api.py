@@ -240,8 +240,10 @@ class Plan:
 
     @property
     def n_tile_pairs(self):
-        """Thread blocks per (batch, head) of a block-sparse launch: pairs of 128-row query tiles."""
-        return ((self.N + 127) // 128 + 1) // 2
+        """Thread blocks per (batch, head) of a block-sparse launch: pairs of query tiles (a tile holds two
+        blocks of up to 64 tokens, or one larger block)."""
+        per_tile = 2 if self.block <= 64 else 1
+        return ((self.NB + per_tile - 1) // per_tile + 1) // 2
 
     def build_block_mask(self, ridx, block_mask=None, row_ptr=None, col_idx=None, nnz=None, tile_pairs=None,
                          want_tile_pairs=False):

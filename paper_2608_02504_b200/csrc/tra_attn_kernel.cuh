@@ -312,7 +312,9 @@ struct Cfg {
   static constexpr int kBlocksPerCta = 2 * kGroups;
   static constexpr int kQTileBytes = kTileM * D * 2;
   static constexpr int kSlotBytes = BN * D * 2;
-  static constexpr int kSlots = (D == 128 && BN == 128) ? 5 : 6;
+  static constexpr int kSlots = (D == 128 && BN > 96) ? 5 : 6;
+  static constexpr int kChunks = (BN + 31) / 32;               // 32-key chunks of a score row
+  static constexpr int kCols = kChunks * 32;
   static constexpr int kKSlots = 3;                            // block-sparse launches: K ring / V ring
   static constexpr int kVSlots = kSlots - kKSlots;
   static constexpr int kAtoms = D / 64;                        // 64-column swizzle atoms per row
@@ -357,15 +359,21 @@ struct TokenMaskArgs {
 // kDense: every query block attends to every key block (no block list; row_ptr is not read).
 // kLse: the caller wants lse from a launch without entropy; the row sum of the unrounded
 // probabilities is then accumulated next to the bf16-rounded one (kEntropy always does).
-template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense, bool kLse>
+template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense, bool kLse, bool kAny>
 __global__ void __launch_bounds__(kThreads, 1)
 tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                 const __grid_constant__ CUtensorMap map_v, __nv_bfloat16* __restrict__ O,
                 float* __restrict__ entropy, float* __restrict__ lse,
                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                 const int32_t* __restrict__ tile_pairs, int N, int NB, float scale_log2,
-                int* __restrict__ status, TokenMaskArgs tm) {
+                int* __restrict__ status, TokenMaskArgs tm, int blk_arg) {
   using C = Cfg<D, BN>;
+  static_assert(!(kAny && kTokenMask), "the token mask needs blocks of whole 16-key slices");
+  // kAny: blocks of blk <= BN tokens (BN = blk rounded up to a multiple of 16).  A key tile is still BN rows,
+  // loaded from row v * blk: its last BN - blk rows belong to the next block and are masked as columns; a query
+  // tile holds kGroups blocks in its first tile_rows rows and the rest of its 128 rows are computed and dropped.
+  const int blk = kAny ? blk_arg : BN;
+  const int tile_rows = C::kGroups * blk;
   constexpr bool kExact = kEntropy || kLse;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -378,7 +386,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   // The two 128-row query tiles of this CTA: consecutive ones, or the pair the block-mask call chose
   // (tiles with similar block lists share a CTA, so that few key blocks serve one tile only).
   // A missing tile (index -1) has no rows and no list.
-  const int NT = (N + kTileM - 1) / kTileM;
+  const int NT = (N + tile_rows - 1) / tile_rows;
   int tile0 = 2 * (int)blockIdx.x, tile1 = 2 * (int)blockIdx.x + 1;
   if (!kDense && tile_pairs != nullptr) {
     const int32_t* pr = tile_pairs + ((size_t)bh * gridDim.x + blockIdx.x) * 2;
@@ -509,13 +517,13 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       for (int k = 0; k < 2; ++k)
         for (int a = 0; a < C::kAtoms; ++a)
           tma_load_3d(smem_u32(sQ + k * C::kQTileBytes + a * C::kQAtomBytes), &map_q, qbar, a * 64,
-                      max(tile_index(k), 0) * kTileM, bh);      // a missing tile loads rows nobody uses
+                      max(tile_index(k), 0) * tile_rows, bh);      // a missing tile loads rows nobody uses
       bool alive = true;
       auto load_tile = [&](const CUtensorMap* map, int slot, int v) {
         const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
         mbar_expect_tx(fbar, C::kSlotBytes);
         for (int a = 0; a < C::kAtoms; ++a)
-          tma_load_3d(smem_u32(sKV + slot * C::kSlotBytes + a * C::kKVAtomBytes), map, fbar, a * 64, v * BN, bh);
+          tma_load_3d(smem_u32(sKV + slot * C::kSlotBytes + a * C::kKVAtomBytes), map, fbar, a * 64, v * blk, bh);
       };
       if constexpr (kDense) {
         // Loads go K0, V0, K1, V1, ... into consecutive slots.  The MMA warp hands slots back in
@@ -646,11 +654,11 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         const uint32_t pa = tmem + buf * 128;
         const uint32_t started = (pv_started >> k) & 1u;
 #pragma unroll
-        for (int half = 0; half < BN / 64; ++half) {
+        for (int half = 0; half < (BN + 63) / 64; ++half) {
           if (!mbar_wait(p_ready_bar + (buf * 2 + half) * 8, parity, abort_flag, status)) return false;
           tc_fence_after();
 #pragma unroll
-          for (int kk = half * 4; kk < half * 4 + 4; ++kk)
+          for (int kk = half * 4; kk < half * 4 + 4 && kk < BN / 16; ++kk)
             tc_mma_ts(d, pa + kk * 8, va + kk * (2048 >> 4), kHi, kIdescPV, kk > 0 ? 1u : started);
         }
         pv_started |= 1u << k;
@@ -834,9 +842,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // ================================================================== softmax + epilogue
     const int k = warp >> 2;                         // query tile
     const int r = tid & (kTileM - 1);                // row inside the tile
-    const int row = tile_index(k) * kTileM + r;                  // negative for a missing tile
-    const bool row_valid = row >= 0 && row < N;
-    const int g_own = k * C::kGroups + r / BN;
+    const int row = tile_index(k) * tile_rows + r;               // meaningless for a missing tile (index -1)
+    const bool row_valid = tile_index(k) >= 0 && r < tile_rows && row < N;
+    const int g_own = k * C::kGroups + min(r / blk, C::kGroups - 1);
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t t_o = tmem + lane_base + 256 + k * 128;
 
@@ -846,7 +854,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     bool tm_row = false;
     int qx = 0, qy = 0, qt = 0;
     const int32_t* th_row = nullptr;
-    if (kTokenMask && row >= 0 && row < tm.n_video) {
+    if (kTokenMask && row_valid && row < tm.n_video) {
       const uint32_t c = tm.coord_packed[row];
       qx = tra_coord_x(c);
       qy = tra_coord_y(c);
@@ -887,7 +895,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           job_prev = job;
           if (C::kGroups > 1) active = (own_bits & low) != 0;
         }
-        const int col_limit = min(BN, N - v * BN);
+        const int col_limit = min(blk, N - v * blk);
         const uint32_t t_s = tmem + lane_base + buf * 128;
 
         if (!mbar_wait_warp(smem_u32(&ctl->s_full[k][buf]), (s_seen >> buf) & 1u, abort_flag, status)) {
@@ -898,17 +906,26 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         tc_fence_after();
 
         // the whole S row of this thread, straight into registers (one load latency)
-        uint32_t sb[BN];
+        uint32_t sb[C::kCols];
 #pragma unroll
-        for (int c = 0; c < BN / 32; ++c) tmem_ld32(t_s + c * 32, &sb[c * 32]);
+        for (int c = 0; c < C::kChunks; ++c) tmem_ld32(t_s + c * 32, &sb[c * 32]);
         tmem_wait_ld(&sb[0]);
 #pragma unroll
-        for (int c = 1; c < BN / 32; ++c) reg_fence32(&sb[c * 32]);
+        for (int c = 1; c < C::kChunks; ++c) reg_fence32(&sb[c * 32]);
 
-        if (col_limit < BN) {          // ragged last key block: columns >= col_limit do not exist
+        // Columns >= col_limit do not exist: the ragged last key block, and with kAny the tail of every key tile
+        // (rows of the next block, and tensor-memory columns past BN that no MMA wrote).  Only the last 32
+        // columns can be concerned unless the block is the ragged last one.
+        if (col_limit < C::kCols) {
+          if (col_limit >= C::kCols - 32) {
 #pragma unroll
-          for (int j = 0; j < BN; ++j)
-            if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
+            for (int j = C::kCols - 32; j < C::kCols; ++j)
+              if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
+          } else {
+#pragma unroll
+            for (int j = 0; j < C::kCols; ++j)
+              if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
+          }
         }
         if (kTokenMask && tm_row && active && v * BN < tm.n_video) {
           // keys outside this query's disk at their frame distance do not exist for it (Eq. 15);
@@ -982,11 +999,11 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (active) {
           float mx0 = __uint_as_float(sb[0]), mx1 = __uint_as_float(sb[1]);
 #pragma unroll
-          for (int j = 2; j + 3 < BN; j += 4) {
+          for (int j = 2; j + 3 < C::kCols; j += 4) {
             mx0 = fmax3(mx0, __uint_as_float(sb[j]), __uint_as_float(sb[j + 1]));
             mx1 = fmax3(mx1, __uint_as_float(sb[j + 2]), __uint_as_float(sb[j + 3]));
           }
-          mx0 = fmax3(mx0, __uint_as_float(sb[BN - 2]), __uint_as_float(sb[BN - 1]));
+          mx0 = fmax3(mx0, __uint_as_float(sb[C::kCols - 2]), __uint_as_float(sb[C::kCols - 1]));
           const float mx = fmaxf(mx0, mx1);
           if (kTokenMask) row_on = mx > -1e29f;
           const float m_blk = mx * scale_log2;
@@ -1037,7 +1054,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           float l_lo = 0.f, l_hi = 0.f;
           uint64_t a2 = 0ull, e2 = 0ull;                 // pairs of partial sums
 #pragma unroll
-          for (int c = 0; c < BN / 32; ++c) {
+          for (int c = 0; c < C::kChunks; ++c) {
             uint32_t pk[16];
             if (active) {
 #pragma unroll
@@ -1067,7 +1084,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
               for (int j = 0; j < 16; ++j) pk[j] = 0u;
             }
             tmem_st16(t_s + c * 16, pk);
-            if (c & 1) {                      // a 64-key half of P is complete
+            if ((c & 1) || c == C::kChunks - 1) {   // a 64-key half of P (the last may be shorter) is complete
               tmem_wait_st();
               tc_fence_before();
               __syncwarp();
@@ -1188,7 +1205,7 @@ int make_map(CUtensorMap* map, const void* base, int d, int N, long long BH, int
   return r == CUDA_SUCCESS ? TRA_OK : TRA_ERR_CUDA;
 }
 
-template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense, bool kLse>
+template <int D, int BN, bool kEntropy, bool kTokenMask, bool kDense, bool kLse, bool kAny = false>
 int launch(const tra_attn_args& a) {
   using C = Cfg<D, BN>;
   const tra_plan_t* plan = a.plan;
@@ -1197,15 +1214,16 @@ int launch(const tra_attn_args& a) {
   if ((rc = make_map(&mq, a.Q, D, plan->S, a.BH, kTileM)) != TRA_OK) return rc;
   if ((rc = make_map(&mk, a.K, D, plan->S, a.BH, BN)) != TRA_OK) return rc;
   if ((rc = make_map(&mv, a.V, D, plan->S, a.BH, BN)) != TRA_OK) return rc;
-  auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense, kLse>;
+  auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense, kLse, kAny>;
   TokenMaskArgs tm = {plan->d_boxes, plan->d_slice, plan->d_coord_packed, plan->d_theta, a.ridx,
                       plan->N,       plan->cfg.T,   plan->n_radii};
   TRA_CUDA_CHECK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes));
-  const int n_pairs = (plan->S + 2 * kTileM - 1) / (2 * kTileM);
+  const int tile_rows = C::kGroups * (kAny ? plan->cfg.block : BN);      // query rows a tile really holds
+  const int n_pairs = ((plan->S + tile_rows - 1) / tile_rows + 1) / 2;
   dim3 grid((unsigned)n_pairs, (unsigned)a.BH);
   kern<<<grid, kThreads, C::kSmemBytes, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.O, a.entropy, a.lse, a.row_ptr,
                                                     a.col_idx, a.tile_pairs, plan->S, plan->NB,
-                                                    a.sm_scale * kLog2e, plan->d_status, tm);
+                                                    a.sm_scale * kLog2e, plan->d_status, tm, plan->cfg.block);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }
@@ -1222,6 +1240,18 @@ int launch_shape(const tra_attn_args& a) {
   if (a.row_ptr == nullptr)
     return want_lse ? launch<D, BN, false, false, true, true>(a) : launch<D, BN, false, false, true, false>(a);
   return want_lse ? launch<D, BN, false, false, false, true>(a) : launch<D, BN, false, false, false, false>(a);
+}
+
+// Blocks of any size in (BN - 16, BN] (the paper's 40 .. 120-token blocks): dense and block-sparse launches; the
+// token mask inside blocks needs whole 16-key slices and is refused.
+template <int D, int BN>
+int launch_shape_any(const tra_attn_args& a) {
+  const bool want_lse = a.lse != nullptr;
+  if (a.ridx != nullptr) return TRA_ERR_UNSUPPORTED;
+  if (a.entropy != nullptr) return launch<D, BN, true, false, true, false, true>(a);
+  if (a.row_ptr == nullptr)
+    return want_lse ? launch<D, BN, false, false, true, true, true>(a) : launch<D, BN, false, false, true, false, true>(a);
+  return want_lse ? launch<D, BN, false, false, false, true, true>(a) : launch<D, BN, false, false, false, false, true>(a);
 }
 
 }  // namespace

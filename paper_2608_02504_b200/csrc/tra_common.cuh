@@ -81,6 +81,10 @@ __host__ __device__ inline int tra_field_row_words(int W) { return 4 * (((W + 4)
     if (_e != cudaSuccess) return TRA_ERR_CUDA;   \
   } while (0)
 
+// Query blocks per 128-row query tile of the attention launches, for blocks of more than 32 tokens: a tile holds two
+// blocks of up to 64 tokens or one larger block (its first G * b rows are used).
+inline int tra_blocks_per_tile(int block) { return block <= 64 ? 2 : 1; }
+
 // Plan time: the coarse table of the two-round radius search (tra_radius.cu).
 int tra_build_coarse_table(const uint32_t* counts, uint32_t* coarse, long long cells, int n_radii, int* status,
                            cudaStream_t stream);

@@ -43,7 +43,8 @@ HostPassLayout make_layout(const tra_plan_t* plan, int group) {
   L.row_ptr = take((g * NB + 1) * 4);
   L.col_idx = take(g * NB * NB * 4);
   L.nnz = take(8);
-  L.pairs = take(g * (((S + 127) / 128 + 1) / 2) * 2 * 4);
+  const size_t G = (size_t)tra_blocks_per_tile(plan->cfg.block), NT = (NB + G - 1) / G;    // query tiles
+  L.pairs = take(g * ((NT + 1) / 2) * 2 * 4);
   L.total = off;
   return L;
 }

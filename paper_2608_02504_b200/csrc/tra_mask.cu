@@ -658,7 +658,7 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   const int NB = plan->NB, T = plan->cfg.T;
   const long long BH = (long long)B * heads;
   if (NB > 65535 || BH > 65535) return TRA_ERR_UNSUPPORTED;
-  if (tile_pairs && 128 % plan->cfg.block != 0) return TRA_ERR_UNSUPPORTED;   // no attention launch, no query tiles
+  if (tile_pairs && plan->cfg.block <= 32) return TRA_ERR_UNSUPPORTED;   // no attention launch, no query tiles
   const long long rows = BH * NB;
 
   const int H = plan->cfg.H, W = plan->cfg.W;
@@ -675,9 +675,9 @@ extern "C" int tra_build_block_mask(const tra_plan_t* plan, const uint16_t* ridx
   int G = 1, NT = 0, frame_tiles = 0;
   size_t pair_smem = 0;
   if (tile_pairs) {
-    // query tiles of the attention launch: 128 rows = G blocks
+    // query tiles of the attention launch: G blocks each
     const int b = plan->cfg.block;
-    G = 128 / b;
+    G = tra_blocks_per_tile(b);
     NT = (NB + G - 1) / G;
     // tiles per frame, rounded: the tile one frame ahead of u is u + frame_tiles or a neighbour of it
     const long long tile_tokens = (long long)b * G;

@@ -269,11 +269,85 @@ def test_random_geometries_integer_stages_and_token_mask(cfg):
     plan.close()
 
 
-@pytest.mark.parametrize("block", [48, 80])
-def test_block_sizes_that_do_not_divide_the_query_tile(block):
-    """Block sizes like the paper's 40 .. 120 have a block mask (bit for bit against the oracle) but no
-    attention launch, hence no query tiles to pair: asking for the tile-pair table is refused before
-    anything runs, and the mask buffers stay untouched."""
+# Blocks of the paper's sizes (Appendix, hyper-parameter tables: 40, 48, 72, 90, 120 tokens; tiles used as
+# blocks) and a few more, each with a tile shape that holds exactly one block or that blocks straddle.
+PAPER_BLOCK_CASES = [
+    (40, dict(T=3, H=10, W=16, tile_h=5, tile_w=8)),       # 5 x 8 tiles = blocks, N = 480
+    (48, dict(T=4, H=12, W=16, tile_h=6, tile_w=8)),       # N = 768
+    (56, dict(T=3, H=9, W=14, tile_h=4, tile_w=8)),        # blocks straddle tiles, ragged last block (N = 378)
+    (72, dict(T=3, H=16, W=18, tile_h=8, tile_w=9)),       # N = 864
+    (90, dict(T=4, H=9, W=20, tile_h=9, tile_w=10)),       # the 9 x 10 tiles of a 45 x 80 frame, N = 720
+    (90, dict(T=3, H=11, W=23, tile_h=9, tile_w=10)),      # clipped edge tiles, ragged last block (N = 759)
+    (100, dict(T=3, H=10, W=20, tile_h=10, tile_w=10)),    # N = 600
+    (120, dict(T=5, H=10, W=24, tile_h=10, tile_w=12)),    # N = 1200
+    (33, dict(T=2, H=11, W=9, tile_h=4, tile_w=4)),        # the smallest block the attention calls take
+]
+
+
+@pytest.mark.parametrize("block,grid", PAPER_BLOCK_CASES, ids=[f"b{b}-{g['T']}x{g['H']}x{g['W']}" for b, g in PAPER_BLOCK_CASES])
+def test_paper_block_sizes_whole_path(block, grid):
+    """Dense attention + entropy, block vote, tile pairs and block-sparse attention with blocks that are neither
+    64 nor 128 tokens: every row against the oracle, lists bit for bit."""
+    cfg = common.small_config(grid["T"], grid["H"], grid["W"], heads=2, head_dim=128, block=block,
+                              tile_h=grid["tile_h"], tile_w=grid["tile_w"], seed=300 + block, s_lo=0.2, s_hi=5.0)
+    geo = common.oracle_geometry(cfg)
+    plan = make_plan(cfg)
+    Q, K, V = tile_major_inputs(cfg, plan)
+    O, H, lse = plan.entropy_attn(Q, K, V, want_lse=True)
+    O2, _, _ = plan.entropy_attn(Q, K, V, want_entropy=False)
+    plan.check_status()
+    Qb, Kb, Vb = (workloads.bf16_bits(x)[0] for x in (Q, K, V))
+    rows = np.arange(geo.N)
+    dense = [oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows) for h in range(cfg["heads"])]
+    for h in range(cfg["heads"]):
+        common.assert_output(O[0, h], dense[h]["O"], f"dense head {h}")
+        common.assert_output(O2[0, h], dense[h]["O"], f"dense (no entropy) head {h}")
+        assert np.abs(H[0, h].cpu().numpy().astype(np.float64) - dense[h]["H_def"]).max() <= common.ENTROPY_ATOL
+        assert np.abs(lse[0, h].cpu().numpy().astype(np.float64) - dense[h]["lse"]).max() <= 1e-3
+    # the pipeline's own radii, then two synthetic kinds (whole blocks sharp or diffuse: empty and full rows)
+    _, _, ridx_t = plan.budget_radius(H)
+    kinds = [("pipeline", ridx_t.cpu().numpy().view(np.uint16)[0])]
+    kinds += [(k, random_ridx(geo, cfg["heads"], np.random.default_rng(41), k)) for k in ("blocky", "small")]
+    for kind, ridx in kinds:
+        ridx_t = torch.from_numpy(np.ascontiguousarray(ridx).view(np.int16)).to(DEV)[None]
+        mask, row_ptr, col_idx, nnz, pairs = plan.build_block_mask(ridx_t, want_tile_pairs=True)
+        Os, lse_s = plan.sparse_attn(Q, K, V, row_ptr, col_idx, want_lse=True)
+        Op, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, tile_pairs=pairs)
+        plan.check_status()
+        assert torch.equal(Os, Op), kind                              # the pairing only moves time
+        per_tile = 2 if block <= 64 else 1
+        NT = (geo.NB + per_tile - 1) // per_tile
+        for h in range(cfg["heads"]):
+            used = pairs[h].flatten().cpu().numpy()
+            assert sorted(used[used >= 0].tolist()) == list(range(NT)), kind      # a perfect matching of the tiles
+            ref_mask = oracle.block_vote(geo.coord, geo.T, geo.block, geo.theta, ridx[h])
+            assert np.array_equal(mask.cpu().numpy()[0, h], ref_mask), kind
+            vis = oracle.visible_rows(geo.coord, geo.T, geo.block, geo.theta, ridx[h], rows, ref_mask[rows // block], 0)
+            ref = oracle.attention_rows(Qb[h], Kb[h], Vb[h], common.scale_of(cfg), rows, vis)
+            common.assert_output(Os[0, h], ref["O"], f"sparse ({kind}) head {h}")
+            empty = ~vis.any(axis=1)
+            assert np.all(Os[0, h].float().cpu().numpy()[empty] == 0)
+            got_lse = lse_s[0, h].cpu().numpy().astype(np.float64)
+            assert np.all(np.isneginf(got_lse[empty]))
+            if (~empty).any():
+                assert np.abs(got_lse[~empty] - ref["lse"][~empty]).max() <= 1e-3
+    # every block retained: the sparse launch gives the dense launch's bits
+    full = torch.ones(1, cfg["heads"], geo.NB, geo.NB, dtype=torch.uint8)
+    rp, ci = oracle.csr_from_block_mask(full.numpy()[0])
+    Of, _ = plan.sparse_attn(Q, K, V, torch.from_numpy(rp.astype(np.int32)).to(DEV), torch.from_numpy(ci).to(DEV))
+    assert torch.equal(Of, O2)
+    # the token mask inside blocks needs whole 16-key slices: refused, nothing runs
+    with pytest.raises(api().TraError) as err:
+        plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx_t)
+    assert err.value.code == api().TRA_ERR_UNSUPPORTED
+    plan.check_status()
+    plan.close()
+
+
+def test_small_blocks_have_a_mask_but_no_attention_launch():
+    """Blocks of 32 tokens or fewer: the block mask is built (bit for bit against the oracle), the attention calls
+    and the tile-pair table are refused before anything runs, and the mask buffers stay untouched."""
+    block = 24
     cfg = common.small_config(4, 12, 20, heads=2, head_dim=128, block=block, tile_h=4, tile_w=8, seed=85)
     geo = common.oracle_geometry(cfg)
     ridx = random_ridx(geo, cfg["heads"], np.random.default_rng(21), "entropy")
@@ -287,6 +361,10 @@ def test_block_sizes_that_do_not_divide_the_query_tile(block):
     sentinel = torch.full((1, cfg["heads"], geo.NB, geo.NB), 7, dtype=torch.uint8, device=DEV)
     with pytest.raises(api().TraError) as err:
         plan.build_block_mask(ridx_t, block_mask=sentinel, want_tile_pairs=True)
+    assert err.value.code == api().TRA_ERR_UNSUPPORTED
+    Q, K, V = tile_major_inputs(cfg, plan)
+    with pytest.raises(api().TraError) as err:
+        plan.entropy_attn(Q, K, V)
     assert err.value.code == api().TRA_ERR_UNSUPPORTED
     torch.cuda.synchronize()
     assert bool((sentinel == 7).all())
