@@ -562,7 +562,11 @@ def run_sweeps(api, cfg, plan, dev, bufs, t_plain, peak_tf):
     for th, tw in ((8, 16), (16, 8), (4, 32), (1, cfg["W"])):
         out["tile_shape"].append({"tile": [th, tw], **own_pass(api, dict(cfg, tile_h=th, tile_w=tw), Qr, Kr, Vr,
                                                                peak_tf)})
-    for b, (th, tw) in ((128, (8, 16)), (64, (8, 8))):
+    # 128 and 64, then the paper's block sizes as tiles of the 45 x 80 frame (Appendix, block-size table)
+    for b, (th, tw) in ((128, (8, 16)), (64, (8, 8)), (120, (15, 8)), (90, (9, 10)), (72, (9, 8)), (48, (3, 16)),
+                        (40, (5, 8))):
+        if b not in (128, 64) and (cfg["H"] % th or cfg["W"] % tw):     # tiles used as blocks must tile the frame
+            continue
         out["block_size"].append({"block": b, "tile": [th, tw],
                                   **own_pass(api, dict(cfg, block=b, tile_h=th, tile_w=tw), Qr, Kr, Vr, peak_tf)})
     return out
@@ -575,7 +579,7 @@ def own_pass(api, cfg, Qr, Kr, Vr, peak_tf):
     O, H, _ = plan.entropy_attn(Q, K, V)
     t_plain = time_ms(lambda: plan.entropy_attn(Q, K, V, O=O, want_entropy=False), 1, 0)
     plan.close()
-    return sparse_layer(api, cfg, Q, K, V, O, H, t_plain, peak_tf, reps=2)
+    return {"dense_plain_ms": round(t_plain, 3), **sparse_layer(api, cfg, Q, K, V, O, H, t_plain, peak_tf, reps=2)}
 
 
 def run_schedule(cfg, plan, dev, bufs, n_steps, n_warm, refresh_every=0, entropy_last_only=False):

@@ -32,6 +32,9 @@ def main():
         (common.small_config(6, 16, 24, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16, seed=80,
                              s_lo=0.2, s_hi=5.0), 100),
         (common.small_config(3, 7, 10, heads=3, head_dim=64, block=64, tile_h=4, tile_w=4, seed=78), 50),
+        # blocks that are neither 64 nor 128 tokens (no token mask inside blocks for these)
+        (common.small_config(3, 11, 23, heads=2, head_dim=128, block=90, tile_h=9, tile_w=10, seed=82), 0),
+        (common.small_config(3, 10, 16, heads=2, head_dim=128, block=40, tile_h=5, tile_w=8, seed=83), 30),
     ]
     out = []
     for cfg, n_text in cases:
@@ -44,8 +47,9 @@ def main():
         budget, radius, ridx = plan.budget_radius(H)
         mask, row_ptr, col_idx, nnz, pairs = plan.build_block_mask(ridx, want_tile_pairs=True)
         Os, lse_s = plan.sparse_attn(Q, K, V, row_ptr, col_idx, tile_pairs=pairs, want_lse=True)
-        Ot, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx, tile_pairs=pairs)
-        Oe, _ = plan.sparse_attn(Q, K, V, None, None, ridx=ridx)
+        token_mask = cfg["block"] in (64, 128)
+        Ot, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx if token_mask else None, tile_pairs=pairs)
+        Oe, _ = plan.sparse_attn(Q, K, V, None, None, ridx=ridx) if token_mask else (Ot, None)
         back = plan.tile_major_scatter(Os)
         status = plan.status()
         # a list that overflows its buffer, and candidate indices past the table: both are clamped
@@ -55,7 +59,7 @@ def main():
         status_overflow = plan.status()
         wild = torch.full_like(ridx, -1)
         mw, rpw, ciw, _ = plan.build_block_mask(wild)
-        Ow, _ = plan.sparse_attn(Q, K, V, rpw, ciw, ridx=wild)
+        Ow, _ = plan.sparse_attn(Q, K, V, rpw, ciw, ridx=wild if token_mask else None)
         status_wild = plan.status()
         # a list whose offsets run backwards (no entry is read: every row comes out empty); only the
         # bounds-checking build notices
