@@ -884,10 +884,12 @@ def test_batch_and_side_stream():
     plan.close()
 
 
-def test_host_pipeline_matches_device_path():
+@pytest.mark.parametrize("cfg", [dict(CFG_MID128, heads=5),
+                                 common.small_config(4, 9, 20, heads=5, head_dim=128, block=90, tile_h=9, tile_w=10,
+                                                     seed=87, s_lo=0.2, s_hi=5.0)], ids=["mid128", "b90"])
+def test_host_pipeline_matches_device_path(cfg):
     """The head-group pipeline over pinned host tensors (copies overlapped with kernels) returns the
     bits of the one-shot device path, with a ragged last group and with one group."""
-    cfg = dict(CFG_MID128, heads=5)
     plan = make_plan(cfg)
     Qr, Kr, Vr = workloads.make_qkv(cfg, "cuda")
     Q, K, V = (plan.tile_major_gather(x) for x in (Qr, Kr, Vr))
