@@ -68,8 +68,8 @@ typedef struct {
   int T, H, W;         /* latent grid (Section 2.1); 1 <= T,H,W <= 1023                          */
   int head_dim;        /* d: 64 or 128                                                          */
   int block;           /* b of Algorithm 1: 16..128 for the budget/radius/mask calls; the        */
-                       /* attention calls take 33..128 with head_dim 128 (64 or 128 with        */
-                       /* head_dim 64); the token mask inside blocks (ridx) needs 64 or 128     */
+                       /* attention calls take 33..128; the token mask inside blocks (ridx)     */
+                       /* needs 64 or 128                                                       */
   int tile_h, tile_w;  /* tile shape of the tile-major order (Section 3.3)                       */
   double tau;          /* target attention mass of Eq. 4, in (0, 1]                              */
   double gamma;        /* temporal decay rate of Eq. 10, >= 0                                    */

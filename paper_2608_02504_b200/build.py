@@ -19,7 +19,7 @@ LIB = os.path.join(HERE, "libtra_b200.so")
 LIB_DEBUG = os.path.join(HERE, "libtra_b200_debug.so")
 SOURCES = ["tra_plan.cu", "tra_radius.cu", "tra_mask.cu", "tra_attn.cu", "tra_attn_d128_b128.cu",
            "tra_attn_d64_b64.cu", "tra_attn_d64_b128.cu", "tra_attn_d128_b64.cu", "tra_host.cu"] + \
-          [f"tra_attn_d128_any{bn}.cu" for bn in (48, 64, 80, 96, 112, 128)]
+          [f"tra_attn_d{d}_any{bn}.cu" for d in (128, 64) for bn in (48, 64, 80, 96, 112, 128)]
 
 
 def _headers():

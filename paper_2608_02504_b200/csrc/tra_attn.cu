@@ -21,15 +21,16 @@ int attn_dispatch(const tra_plan_t* plan, const void* Q, const void* K, const vo
   if (d == 64 && b == 64) return tra_attn_launch_d64_b64(a);
   if (d == 64 && b == 128) return tra_attn_launch_d64_b128(a);
   if (d == 128 && b == 64) return tra_attn_launch_d128_b64(a);
-  if (d == 128 && b > 32 && b <= 128) {      // any other block size: key tiles of ceil(b / 16) * 16 rows
-    switch ((b + 15) / 16) {
-      case 3: return tra_attn_launch_d128_any48(a);
-      case 4: return tra_attn_launch_d128_any64(a);
-      case 5: return tra_attn_launch_d128_any80(a);
-      case 6: return tra_attn_launch_d128_any96(a);
-      case 7: return tra_attn_launch_d128_any112(a);
-      default: return tra_attn_launch_d128_any128(a);
-    }
+  if (b > 32 && b <= 128) {      // any other block size: key tiles of ceil(b / 16) * 16 rows
+    const int w = (b + 15) / 16;
+    if (d == 128)
+      return w == 3 ? tra_attn_launch_d128_any48(a) : w == 4 ? tra_attn_launch_d128_any64(a)
+           : w == 5 ? tra_attn_launch_d128_any80(a) : w == 6 ? tra_attn_launch_d128_any96(a)
+           : w == 7 ? tra_attn_launch_d128_any112(a) : tra_attn_launch_d128_any128(a);
+    if (d == 64)
+      return w == 3 ? tra_attn_launch_d64_any48(a) : w == 4 ? tra_attn_launch_d64_any64(a)
+           : w == 5 ? tra_attn_launch_d64_any80(a) : w == 6 ? tra_attn_launch_d64_any96(a)
+           : w == 7 ? tra_attn_launch_d64_any112(a) : tra_attn_launch_d64_any128(a);
   }
   return TRA_ERR_UNSUPPORTED;
 }

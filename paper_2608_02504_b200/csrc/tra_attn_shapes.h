@@ -26,7 +26,7 @@ int tra_attn_launch_d128_b128(const tra_attn_args& a);
 int tra_attn_launch_d64_b64(const tra_attn_args& a);
 int tra_attn_launch_d64_b128(const tra_attn_args& a);
 int tra_attn_launch_d128_b64(const tra_attn_args& a);
-// head_dim 128, blocks of 33 .. 128 tokens other than 64 and 128: by key-tile width (the block size rounded up to
+// blocks of 33 .. 128 tokens other than 64 and 128: by head_dim and key-tile width (the block size rounded up to
 // a multiple of 16)
 int tra_attn_launch_d128_any48(const tra_attn_args& a);
 int tra_attn_launch_d128_any64(const tra_attn_args& a);
@@ -34,3 +34,9 @@ int tra_attn_launch_d128_any80(const tra_attn_args& a);
 int tra_attn_launch_d128_any96(const tra_attn_args& a);
 int tra_attn_launch_d128_any112(const tra_attn_args& a);
 int tra_attn_launch_d128_any128(const tra_attn_args& a);
+int tra_attn_launch_d64_any48(const tra_attn_args& a);
+int tra_attn_launch_d64_any64(const tra_attn_args& a);
+int tra_attn_launch_d64_any80(const tra_attn_args& a);
+int tra_attn_launch_d64_any96(const tra_attn_args& a);
+int tra_attn_launch_d64_any112(const tra_attn_args& a);
+int tra_attn_launch_d64_any128(const tra_attn_args& a);

@@ -281,14 +281,17 @@ PAPER_BLOCK_CASES = [
     (100, dict(T=3, H=10, W=20, tile_h=10, tile_w=10)),    # N = 600
     (120, dict(T=5, H=10, W=24, tile_h=10, tile_w=12)),    # N = 1200
     (33, dict(T=2, H=11, W=9, tile_h=4, tile_w=4)),        # the smallest block the attention calls take
+    (90, dict(T=3, H=9, W=20, tile_h=9, tile_w=10, head_dim=64)),
+    (40, dict(T=3, H=10, W=16, tile_h=5, tile_w=8, head_dim=64)),
+    (112, dict(T=3, H=14, W=16, tile_h=7, tile_w=16, head_dim=64)),
 ]
 
 
-@pytest.mark.parametrize("block,grid", PAPER_BLOCK_CASES, ids=[f"b{b}-{g['T']}x{g['H']}x{g['W']}" for b, g in PAPER_BLOCK_CASES])
+@pytest.mark.parametrize("block,grid", PAPER_BLOCK_CASES, ids=[f"b{b}-{g['T']}x{g['H']}x{g['W']}-d{g.get('head_dim', 128)}" for b, g in PAPER_BLOCK_CASES])
 def test_paper_block_sizes_whole_path(block, grid):
     """Dense attention + entropy, block vote, tile pairs and block-sparse attention with blocks that are neither
     64 nor 128 tokens: every row against the oracle, lists bit for bit."""
-    cfg = common.small_config(grid["T"], grid["H"], grid["W"], heads=2, head_dim=128, block=block,
+    cfg = common.small_config(grid["T"], grid["H"], grid["W"], heads=2, head_dim=grid.get("head_dim", 128), block=block,
                               tile_h=grid["tile_h"], tile_w=grid["tile_w"], seed=300 + block, s_lo=0.2, s_hi=5.0)
     geo = common.oracle_geometry(cfg)
     plan = make_plan(cfg)
