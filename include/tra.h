@@ -14,7 +14,8 @@
  * are listed frame by frame, tile by tile, row-major inside a tile).  A block is
  * `block` consecutive tile-major positions (Algorithm 1: q = u*b + i, q < N);
  * NB = ceil(N / block).  tra_tile_major_gather / _scatter move tensors between
- * raster order (n = (t*H + y)*W + x) and tile-major order.
+ * raster order (n = (t*H + y)*W + x) and tile-major order.  A plan created with
+ * TRA_ORDER_RASTER takes Q, K, V and O in raster order instead and needs no such pass.
  *
  * Joint text-video attention (Section 3.2, last paragraph; Algorithm 1).  With cfg.n_text > 0 a
  * sequence is the N video tokens followed by n_text text tokens, S = N + n_text; S takes the place
@@ -52,6 +53,14 @@ extern "C" {
 
 /* plan flags */
 #define TRA_KEEP_DIAGONAL 1u /* force block_mask[u][u] = 1 (a token always sees itself, Eq. 15) */
+#define TRA_ORDER_RASTER 2u  /* Q, K, V and O of the attention calls (and of tra_hot_path_host) are in RASTER   */
+                             /* order, n = (t*H + y)*W + x: the kernels fetch every run of 16 tile-major     */
+                             /* positions, which is 16 consecutive raster rows, with a TMA box of its own and */
+                             /* write O rows where they belong, so no gather / scatter pass is needed         */
+                             /* (Section 3.3 reorders explicitly).  entropy, lse, budget, radius, ridx and    */
+                             /* the mask stay in tile-major order: they only travel between this library's    */
+                             /* calls.  Needs W, tile_w and block to be multiples of 16 (else                  */
+                             /* tra_plan_create returns TRA_ERR_UNSUPPORTED).                                 */
 
 /* entropy-to-budget maps */
 #define TRA_BUDGET_UNIFORM 0   /* K = ceil(tau exp(H)): the uniform-support map of Eq. 8 (the paper's choice) */
@@ -77,7 +86,7 @@ typedef struct {
                        /* one must reach full support (may be +inf).  NULL = radius_policy       */
   int n_radii;
   int radius_policy;   /* TRA_RADII_* (used when radii == NULL)                                  */
-  unsigned flags;      /* TRA_KEEP_DIAGONAL                                                      */
+  unsigned flags;      /* TRA_KEEP_DIAGONAL | TRA_ORDER_RASTER                                   */
   int budget_map;      /* TRA_BUDGET_* used by tra_budget_radius                                 */
   int n_text;          /* text tokens that follow the video tokens in every sequence (>= 0)     */
 } tra_config_t;

@@ -97,6 +97,11 @@ int tra_oracle_default_radii(int T, int H, int W, double gamma, int policy, doub
       out[n++] = r;
     }
   }
+  /* The last candidate is the full-support radius: it must cover the diagonal at the largest frame
+   * distance.  In exact arithmetic D*exp(gamma*(T-1)) does; when the diagonal is an integer (D^2 =
+   * diag2) the rounded product r*r*exp(-2*gamma*(T-1)) can fall just below diag2, and the radius is
+   * then moved up by single floating-point steps until it covers. */
+  while (!(out[n - 1] * out[n - 1] * exp(-2.0 * gamma * (double)(T - 1)) >= diag2)) out[n - 1] = nextafter(out[n - 1], INFINITY);
   return n;
 }
 

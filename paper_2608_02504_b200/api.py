@@ -19,6 +19,7 @@ LIB_PATH = os.environ.get("TRA_B200_LIB") or os.path.join(_HERE, "libtra_b200.so
 TRA_OK = 0
 TRA_ERR_INVALID_ARG, TRA_ERR_UNSUPPORTED, TRA_ERR_CAPACITY, TRA_ERR_CUDA, TRA_ERR_TIMEOUT, TRA_ERR_BOUNDS = -1, -2, -3, -4, -5, -6
 TRA_KEEP_DIAGONAL = 1
+TRA_ORDER_RASTER = 2
 TRA_RADII_EXTENDED = 0
 TRA_RADII_LITERAL = 1
 TRA_BUDGET_UNIFORM = 0
@@ -129,7 +130,7 @@ class Plan:
         self.NB = _lib.tra_plan_num_blocks(self._h)
         self.n_radii = _lib.tra_plan_num_radii(self._h)
         self.T, self.H, self.W = T, H, W
-        self.head_dim, self.block = head_dim, block
+        self.head_dim, self.block, self.flags = head_dim, block, flags
 
     @classmethod
     def from_config(cls, cfg: dict, **overrides):
@@ -332,7 +333,9 @@ class HostPipeline:
         self.workspace_bytes = int(_lib.tra_hot_path_host_workspace_bytes(plan._h, self.group))
         self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.dev)
         self._ws_ptr = (self.workspace.data_ptr() + 255) & ~255
-        self.launches_per_group = 11      # 3 gathers, dense, budget, vote + scan + fill + pairing, sparse, scatter
+        # 3 gathers, dense, budget, vote + scan + fill + pairing, sparse, scatter; a raster-order plan has no
+        # gathers and no scatter
+        self.launches_per_group = 7 if plan.flags & TRA_ORDER_RASTER else 11
         self.n_groups = len(self.group_sizes(heads, self.group, self.first_group))
 
     @staticmethod

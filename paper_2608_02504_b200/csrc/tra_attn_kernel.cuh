@@ -366,7 +366,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 float* __restrict__ entropy, float* __restrict__ lse,
                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                 const int32_t* __restrict__ tile_pairs, int N, int NB, float scale_log2,
-                int* __restrict__ status, TokenMaskArgs tm, int blk_arg) {
+                int* __restrict__ status, TokenMaskArgs tm, int blk_arg,
+                const int32_t* __restrict__ slice_raster) {
   using C = Cfg<D, BN>;
   static_assert(!(kAny && kTokenMask), "the token mask needs blocks of whole 16-key slices");
   // kAny: blocks of blk <= BN tokens (BN = blk rounded up to a multiple of 16).  A key tile is still BN rows,
@@ -514,16 +515,33 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (lane == 0) {
       const uint32_t qbar = smem_u32(&ctl->q_full);
       mbar_expect_tx(qbar, 2 * C::kQTileBytes);
-      for (int k = 0; k < 2; ++k)
-        for (int a = 0; a < C::kAtoms; ++a)
-          tma_load_3d(smem_u32(sQ + k * C::kQTileBytes + a * C::kQAtomBytes), &map_q, qbar, a * 64,
-                      max(tile_index(k), 0) * tile_rows, bh);      // a missing tile loads rows nobody uses
+      // Rows [row0, row0 + rows) of the tile-major order into a tile at `dst` (atoms `atom_bytes` apart).  With the
+      // tensors in tile-major order that is one box per 64-column atom.  With the tensors in RASTER order
+      // (slice_raster != NULL) every 16 consecutive tile-major positions are 16 consecutive raster rows, which
+      // start at slice_raster[position / 16]: one box of 16 rows per slice, 2 KB apart in the tile (the swizzle
+      // pattern repeats every 8 rows, so the tile in shared memory is the same either way).
+      auto load_rows = [&](const CUtensorMap* map, uint32_t dst, uint32_t bar, int row0, int rows, int atom_bytes) {
+        if (slice_raster == nullptr) {
+          for (int a = 0; a < C::kAtoms; ++a) tma_load_3d(dst + a * atom_bytes, map, bar, a * 64, row0, bh);
+        } else {
+          int rr[kTileM / 16];
+#pragma unroll
+          for (int j = 0; j < kTileM / 16; ++j) rr[j] = j * 16 < rows ? __ldg(slice_raster + (row0 >> 4) + j) : 0;
+#pragma unroll
+          for (int j = 0; j < kTileM / 16; ++j)
+            if (j * 16 < rows)
+              for (int a = 0; a < C::kAtoms; ++a)
+                tma_load_3d(dst + a * atom_bytes + j * 2048, map, bar, a * 64, rr[j], bh);
+        }
+      };
+      for (int k = 0; k < 2; ++k)      // a missing tile loads rows nobody uses
+        load_rows(&map_q, smem_u32(sQ + k * C::kQTileBytes), qbar, max(tile_index(k), 0) * tile_rows, kTileM,
+                  C::kQAtomBytes);
       bool alive = true;
       auto load_tile = [&](const CUtensorMap* map, int slot, int v) {
         const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
         mbar_expect_tx(fbar, C::kSlotBytes);
-        for (int a = 0; a < C::kAtoms; ++a)
-          tma_load_3d(smem_u32(sKV + slot * C::kSlotBytes + a * C::kKVAtomBytes), map, fbar, a * 64, v * blk, bh);
+        load_rows(map, smem_u32(sKV + slot * C::kSlotBytes), fbar, v * blk, BN, C::kKVAtomBytes);
       };
       if constexpr (kDense) {
         // Loads go K0, V0, K1, V1, ... into consecutive slots.  The MMA warp hands slots back in
@@ -1118,7 +1136,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     if (alive) {
       tc_fence_after();
       const float inv_l = l > 0.f ? 1.f / l : 0.f;
-      __nv_bfloat16* orow = O + ((size_t)bh * N + (row_valid ? row : 0)) * D;
+      // the output row: the query's own position, or its raster row when the tensors are in raster order
+      const int out_row = !row_valid ? 0 : (slice_raster ? __ldg(slice_raster + (row >> 4)) + (row & 15) : row);
+      __nv_bfloat16* orow = O + ((size_t)bh * N + out_row) * D;
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t o_bits[32];
@@ -1211,9 +1231,11 @@ int launch(const tra_attn_args& a) {
   const tra_plan_t* plan = a.plan;
   CUtensorMap mq, mk, mv;
   int rc;
-  if ((rc = make_map(&mq, a.Q, D, plan->S, a.BH, kTileM)) != TRA_OK) return rc;
-  if ((rc = make_map(&mk, a.K, D, plan->S, a.BH, BN)) != TRA_OK) return rc;
-  if ((rc = make_map(&mv, a.V, D, plan->S, a.BH, BN)) != TRA_OK) return rc;
+  const int32_t* slice_raster = (plan->cfg.flags & TRA_ORDER_RASTER) ? plan->d_slice_raster : nullptr;
+  // boxes: a whole tile per 64-column atom, or (raster order) one 16-token run
+  if ((rc = make_map(&mq, a.Q, D, plan->S, a.BH, slice_raster ? 16 : kTileM)) != TRA_OK) return rc;
+  if ((rc = make_map(&mk, a.K, D, plan->S, a.BH, slice_raster ? 16 : BN)) != TRA_OK) return rc;
+  if ((rc = make_map(&mv, a.V, D, plan->S, a.BH, slice_raster ? 16 : BN)) != TRA_OK) return rc;
   auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense, kLse, kAny>;
   TokenMaskArgs tm = {plan->d_boxes, plan->d_slice, plan->d_coord_packed, plan->d_theta, a.ridx,
                       plan->N,       plan->cfg.T,   plan->n_radii};
@@ -1223,7 +1245,8 @@ int launch(const tra_attn_args& a) {
   dim3 grid((unsigned)n_pairs, (unsigned)a.BH);
   kern<<<grid, kThreads, C::kSmemBytes, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.O, a.entropy, a.lse, a.row_ptr,
                                                     a.col_idx, a.tile_pairs, plan->S, plan->NB,
-                                                    a.sm_scale * kLog2e, plan->d_status, tm, plan->cfg.block);
+                                                    a.sm_scale * kLog2e, plan->d_status, tm, plan->cfg.block,
+                                                    slice_raster);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }

@@ -39,6 +39,7 @@ struct tra_plan {
                                   // x0 | y << 10 | t << 20 | 1 << 30 when they are 16 video tokens of
                                   // one frame and one row with x = x0 .. x0 + 15, else 0
   int32_t* d_raster_of_pos;       // [N]
+  int32_t* d_slice_raster;        // TRA_ORDER_RASTER: [S / 16 + 32] raster row of every 16 consecutive positions
   int32_t* d_theta;               // [n_radii][T]
   float* d_radii_f32;             // [n_radii]
   uint32_t* d_counts;             // [T*H*W][n_radii]  (raster-indexed)

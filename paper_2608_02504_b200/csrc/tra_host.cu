@@ -142,14 +142,19 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
     if (!ready) return TRA_ERR_CUDA;
     TRA_CUDA_CHECK(cudaEventRecord(ready, s_in));
     TRA_CUDA_CHECK(cudaStreamWaitEvent(cs, ready, 0));
-    // the pass itself
+    // the pass itself; a raster-order plan reads the staging buffers in place and writes O into the output
+    // staging buffer, so the gather and scatter kernels drop out
+    const bool raster = (plan->cfg.flags & TRA_ORDER_RASTER) != 0;
     int rc;
-    for (int t = 0; t < 3; ++t)
-      if ((rc = tra_tile_major_gather(plan, ws + L.stage_in[b][t], ws + L.qkv[t], n, row_bytes, cs)) != TRA_OK)
-        return rc;
-    if (!(in_free[b] = pool.make())) return TRA_ERR_CUDA;
-    TRA_CUDA_CHECK(cudaEventRecord(in_free[b], cs));
-    const void *Q = ws + L.qkv[0], *K = ws + L.qkv[1], *V = ws + L.qkv[2];
+    if (!raster) {
+      for (int t = 0; t < 3; ++t)
+        if ((rc = tra_tile_major_gather(plan, ws + L.stage_in[b][t], ws + L.qkv[t], n, row_bytes, cs)) != TRA_OK)
+          return rc;
+      if (!(in_free[b] = pool.make())) return TRA_ERR_CUDA;
+      TRA_CUDA_CHECK(cudaEventRecord(in_free[b], cs));
+    }
+    const void *Q = ws + (raster ? L.stage_in[b][0] : L.qkv[0]), *K = ws + (raster ? L.stage_in[b][1] : L.qkv[1]),
+               *V = ws + (raster ? L.stage_in[b][2] : L.qkv[2]);
     if ((rc = tra_entropy_attn(plan, Q, K, V, ws + L.o_dense, (float*)(ws + L.entropy), nullptr, 1, n, sm_scale,
                                cs)) != TRA_OK)
       return rc;
@@ -160,13 +165,19 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
                                    (int32_t*)(ws + L.col_idx), (int64_t)((size_t)n * NB * NB),
                                    (int64_t*)(ws + L.nnz), (int32_t*)(ws + L.pairs), 1, n, cs)) != TRA_OK)
       return rc;
+    if (raster && out_free[b]) TRA_CUDA_CHECK(cudaStreamWaitEvent(cs, out_free[b], 0));
     if ((rc = tra_sparse_attn(plan, Q, K, V, (const int32_t*)(ws + L.row_ptr), (const int32_t*)(ws + L.col_idx),
-                              nullptr, (const int32_t*)(ws + L.pairs), ws + L.o_sparse, nullptr, 1, n, sm_scale,
-                              cs)) != TRA_OK)
+                              nullptr, (const int32_t*)(ws + L.pairs), ws + (raster ? L.stage_out[b] : L.o_sparse),
+                              nullptr, 1, n, sm_scale, cs)) != TRA_OK)
       return rc;
-    if (out_free[b]) TRA_CUDA_CHECK(cudaStreamWaitEvent(cs, out_free[b], 0));
-    if ((rc = tra_tile_major_scatter(plan, ws + L.o_sparse, ws + L.stage_out[b], n, row_bytes, cs)) != TRA_OK)
-      return rc;
+    if (raster) {                       // the last reader of the input staging buffer
+      if (!(in_free[b] = pool.make())) return TRA_ERR_CUDA;
+      TRA_CUDA_CHECK(cudaEventRecord(in_free[b], cs));
+    } else {
+      if (out_free[b]) TRA_CUDA_CHECK(cudaStreamWaitEvent(cs, out_free[b], 0));
+      if ((rc = tra_tile_major_scatter(plan, ws + L.o_sparse, ws + L.stage_out[b], n, row_bytes, cs)) != TRA_OK)
+        return rc;
+    }
     cudaEvent_t done = pool.make();
     if (!done) return TRA_ERR_CUDA;
     TRA_CUDA_CHECK(cudaEventRecord(done, cs));

@@ -102,6 +102,7 @@ static void tra_plan_free(tra_plan* p) {
   cudaFree(p->d_coord_packed);
   cudaFree(p->d_slice);
   cudaFree(p->d_raster_of_pos);
+  cudaFree(p->d_slice_raster);
   cudaFree(p->d_theta);
   cudaFree(p->d_radii_f32);
   cudaFree(p->d_counts);
@@ -176,6 +177,10 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
         double r = (double)D * exp(cfg->gamma * (double)m);
         if (r > radii.back()) radii.push_back(r);
       }
+      // the last one is the full-support radius: when the diagonal is an integer, rounding can leave
+      // r^2 exp(-2 gamma (T-1)) just below its square; the radius then moves up by single steps until it covers
+      while (!(radii.back() * radii.back() * exp(-2.0 * cfg->gamma * (double)(T - 1)) >= diag2))
+        radii.back() = nextafter(radii.back(), INFINITY);
     } else {
       delete p;
       return TRA_ERR_INVALID_ARG;
@@ -296,6 +301,23 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
     for (size_t i = 0; i < n; ++i) field_pos[i] = (uint16_t)(pos_of[per * i] / per);
   }
 
+  // Raster-order attention (TRA_ORDER_RASTER): the raster row at which every run of 16 consecutive tile-major
+  // positions starts.  Needs every such run to be 16 consecutive raster rows (W and the tile width multiples of
+  // 16) and blocks that start on run boundaries; entries past the sequence hold S, a row outside the tensor (the
+  // load of such a run is filled with zeros).
+  std::vector<int32_t> slice_raster;
+  if (cfg->flags & TRA_ORDER_RASTER) {
+    bool runs = cfg->block % 16 == 0 && p->N % 16 == 0;
+    for (int s0 = 0; s0 < p->N && runs; s0 += 16)
+      for (int i = 1; i < 16 && runs; ++i) runs = raster[s0 + i] == raster[s0] + i;
+    if (!runs) {
+      tra_plan_free(p);
+      return TRA_ERR_UNSUPPORTED;
+    }
+    slice_raster.assign((size_t)p->S / 16 + 32, p->S);
+    for (int s0 = 0; s0 < p->S; s0 += 16) slice_raster[s0 / 16] = s0 < p->N ? raster[s0] : s0;   // text stays in place
+  }
+
   // device tables
   const size_t count_elems = (size_t)p->N * nr;
   bool ok = cudaMalloc(&p->d_coord_packed, sizeof(uint32_t) * (p->N + 128)) == cudaSuccess &&
@@ -308,6 +330,8 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
             cudaMalloc(&p->d_boxes, sizeof(tra_block_boxes_t) * p->NB) == cudaSuccess &&
             (!field_pos_fits || cudaMalloc(&p->d_field_pos, sizeof(uint16_t) * field_pos.size()) == cudaSuccess) &&
             cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess &&
+            (slice_raster.empty() ||
+             cudaMalloc(&p->d_slice_raster, sizeof(int32_t) * slice_raster.size()) == cudaSuccess) &&
             cudaStreamCreateWithFlags(&p->pair_stream, cudaStreamNonBlocking) == cudaSuccess &&
             cudaEventCreateWithFlags(&p->pair_fork, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreateWithFlags(&p->pair_join, cudaEventDisableTiming) == cudaSuccess;
@@ -318,6 +342,9 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
                        stream) == cudaSuccess &&
        cudaMemcpyAsync(p->d_raster_of_pos, raster.data(), sizeof(int32_t) * p->N,
                        cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+       (slice_raster.empty() ||
+        cudaMemcpyAsync(p->d_slice_raster, slice_raster.data(), sizeof(int32_t) * slice_raster.size(),
+                        cudaMemcpyHostToDevice, stream) == cudaSuccess) &&
        cudaMemcpyAsync(p->d_theta, p->h_theta, sizeof(int32_t) * nr * T, cudaMemcpyHostToDevice,
                        stream) == cudaSuccess &&
        cudaMemcpyAsync(p->d_radii_f32, radii_f32.data(), sizeof(float) * nr,

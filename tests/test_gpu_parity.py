@@ -928,6 +928,79 @@ def test_host_pipeline_matches_device_path(cfg):
     plan.close()
 
 
+# Grids whose 16-position runs are 16 consecutive raster rows (W and the tile width multiples of 16).
+RASTER_CASES = [
+    ("b128", common.small_config(4, 12, 32, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16, seed=101, s_lo=0.2,
+                                 s_hi=5.0), 0),
+    ("b128 clipped tiles + text", common.small_config(3, 11, 48, heads=2, head_dim=128, block=128, tile_h=8, tile_w=16,
+                                                      seed=102), 70),
+    ("b64 d64", common.small_config(3, 8, 48, heads=2, head_dim=64, block=64, tile_h=4, tile_w=16, seed=103), 0),
+    ("b96", common.small_config(3, 12, 32, heads=2, head_dim=128, block=96, tile_h=6, tile_w=16, seed=104), 0),
+    ("b48 + text", common.small_config(4, 9, 16, heads=2, head_dim=128, block=48, tile_h=3, tile_w=16, seed=105), 20),
+]
+
+
+@pytest.mark.parametrize("name,cfg,n_text", RASTER_CASES, ids=[c[0] for c in RASTER_CASES])
+def test_raster_order_plan_equals_gather_attend_scatter(name, cfg, n_text):
+    """A plan with TRA_ORDER_RASTER reads Q, K, V in raster order through 16-row TMA boxes and writes O in raster
+    order: every launch gives the bits of gather -> the same launch on tile-major tensors -> scatter, and the
+    per-token outputs (entropy, lse), which stay tile-major, are identical."""
+    plan_t = make_plan(cfg, n_text=n_text)
+    plan_r = make_plan(cfg, n_text=n_text, flags=api().TRA_ORDER_RASTER)
+    Qr, Kr, Vr = workloads.make_qkv(cfg, DEV)
+    if n_text:
+        Qr, Kr, Vr = workloads.append_text(Qr, Kr, Vr, cfg, n_text)
+    Qr, Kr, Vr = (x.contiguous() for x in (Qr, Kr, Vr))
+    Q, K, V = (plan_t.tile_major_gather(x) for x in (Qr, Kr, Vr))
+    token_mask = cfg["block"] in (64, 128)
+    # dense + entropy, plain dense
+    O_t, H_t, lse_t = plan_t.entropy_attn(Q, K, V, want_lse=True)
+    O_r, H_r, lse_r = plan_r.entropy_attn(Qr, Kr, Vr, want_lse=True)
+    assert torch.equal(O_r, plan_t.tile_major_scatter(O_t)) and torch.equal(H_r, H_t) and torch.equal(lse_r, lse_t)
+    P_t, _, _ = plan_t.entropy_attn(Q, K, V, want_entropy=False)
+    P_r, _, _ = plan_r.entropy_attn(Qr, Kr, Vr, want_entropy=False)
+    assert torch.equal(P_r, plan_t.tile_major_scatter(P_t))
+    # the integer stages do not depend on the order of Q, K, V
+    _, _, ridx = plan_t.budget_radius(H_t)
+    _, _, ridx_r = plan_r.budget_radius(H_r)
+    assert torch.equal(ridx, ridx_r)
+    mask, row_ptr, col_idx, nnz, pairs = plan_t.build_block_mask(ridx, want_tile_pairs=True)
+    mask_r, row_ptr_r, col_idx_r, nnz_r, pairs_r = plan_r.build_block_mask(ridx, want_tile_pairs=True)
+    assert torch.equal(mask, mask_r) and torch.equal(row_ptr, row_ptr_r) and torch.equal(pairs, pairs_r)
+    # block-sparse, with and without tile pairs, with lse; token mask inside blocks; Eq. 16 without a list
+    S_t, sl_t = plan_t.sparse_attn(Q, K, V, row_ptr, col_idx, tile_pairs=pairs, want_lse=True)
+    S_r, sl_r = plan_r.sparse_attn(Qr, Kr, Vr, row_ptr, col_idx, tile_pairs=pairs, want_lse=True)
+    assert torch.equal(S_r, plan_t.tile_major_scatter(S_t)) and torch.equal(sl_r, sl_t)
+    S2_r, _ = plan_r.sparse_attn(Qr, Kr, Vr, row_ptr, col_idx)
+    assert torch.equal(S2_r, S_r)
+    if token_mask:
+        for rp, ci in ((row_ptr, col_idx), (None, None)):
+            M_t, _ = plan_t.sparse_attn(Q, K, V, rp, ci, ridx=ridx)
+            M_r, _ = plan_r.sparse_attn(Qr, Kr, Vr, rp, ci, ridx=ridx)
+            assert torch.equal(M_r, plan_t.tile_major_scatter(M_t))
+    # the host pipeline of a raster-order plan: no gather, no scatter, same bits
+    host = [t.cpu().pin_memory() for t in (Qr, Kr, Vr)]
+    out = torch.zeros(S_r.shape, dtype=torch.bfloat16).pin_memory()
+    pipe = api().HostPipeline(plan_r, cfg["heads"], group=1)
+    assert pipe.run(host[0], host[1], host[2], out) == 7 * cfg["heads"]
+    torch.cuda.synchronize()
+    assert torch.equal(out, S_r.cpu())
+    plan_t.check_status()
+    plan_r.check_status()
+    plan_t.close()
+    plan_r.close()
+
+
+def test_raster_order_needs_runs_of_sixteen():
+    """W, the tile width and the block size must be multiples of 16 for a raster-order plan."""
+    for kw in (dict(W=24, tile_w=8, block=128), dict(W=32, tile_w=16, block=72), dict(W=40, tile_w=16, block=128)):
+        cfg = common.small_config(3, 8, kw["W"], heads=1, head_dim=128, block=kw["block"], tile_h=4, tile_w=kw["tile_w"])
+        with pytest.raises(api().TraError) as err:
+            make_plan(cfg, flags=api().TRA_ORDER_RASTER)
+        assert err.value.code == api().TRA_ERR_UNSUPPORTED
+        make_plan(cfg).close()
+
+
 def test_largest_supported_sequence():
     """NB = 2048 key blocks (262,144 tokens) is the largest sequence the attention calls take; one
     more block is refused.  One head, sampled rows against the oracle."""

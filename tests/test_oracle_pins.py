@@ -270,6 +270,29 @@ def test_theta_monotone_in_radius_and_delta():
     assert th.max() == (H - 1) ** 2 + (W - 1) ** 2 and np.all(th[-1] == th.max())
 
 
+def test_full_support_radius_covers_frames_with_an_integer_diagonal():
+    """The last candidate of the extended set is the full-support radius: at every frame distance its threshold is
+    the squared frame diagonal, also when the diagonal is an integer (3-4-5, 5-12-13, 8-15-17 grids), where the
+    rounded product D^2 e^{2 gamma (T-1)} e^{-2 gamma (T-1)} can come out a hair below D^2.  On other grids the
+    extended candidates are D e^{gamma m} to the last bit."""
+    for H, W in ((4, 5), (13, 6), (9, 16), (16, 9), (21, 21)):
+        for T in (2, 4, 21, 33):
+            for gamma in (0.0513, 0.3, 0.6, 0.95, 2.0):
+                radii = oracle.default_radii(T, H, W, gamma)
+                th = oracle.theta_table(radii, T, H, W, gamma)
+                diag2 = (H - 1) ** 2 + (W - 1) ** 2
+                assert np.all(np.diff(radii) > 0)
+                assert np.all(th[-1] == diag2), (H, W, T, gamma)
+                assert oracle.grid_count_brute(T, H, W, th[-1], 0, 0, 0) == T * H * W
+                D = math.ceil(math.sqrt(diag2))
+                want = D * math.exp(gamma * (T - 1))
+                assert radii[-1] == want or 0 < radii[-1] - want <= 4 * np.spacing(want)
+    T, H, W, gamma = 21, 45, 80, 0.6
+    radii = oracle.default_radii(T, H, W, gamma)
+    D = math.ceil(math.sqrt(44 ** 2 + 79 ** 2))
+    assert np.array_equal(radii[D + 1:], [D * math.exp(gamma * m) for m in range(1, T)])
+
+
 # ----------------------------------------------------------------------------- radius
 def test_radius_selection_minimal_and_sufficient():
     g = oracle.geometry(4, 8, 8, 4, 4, 64, 0.6, 0.9)
