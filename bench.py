@@ -294,7 +294,20 @@ def run_ours(args):
 
     sampler = make_sampler(local)
     sampler.start()                     # started early; only samples of the timed region count
-    plan = api.Plan.from_config(cfg)
+    # The timed step gathers Q, K, V into tile-major order and scatters O back, as the paper does.  With
+    # --raster (and a grid that allows it) the step runs on the raster-order tensors instead: the kernels fetch
+    # 16-token runs through TMA boxes of their own and there is no gather / scatter pass.  That saves the two
+    # layout passes and costs more in the attention launches (sixteen small boxes per tile instead of two), so it
+    # is not the default; `stages.raster_order` has both launches' times either way.  plan_tm is the plan for
+    # tile-major tensors, which the measurements after the timed region use.
+    plan_tm = api.Plan.from_config(cfg)
+    plan, raster = plan_tm, False
+    if args.raster:
+        try:
+            plan = api.Plan.from_config(cfg, flags=api.TRA_ORDER_RASTER)
+            raster = True
+        except api.TraError:
+            pass
     Qr, Kr, Vr = workloads.make_qkv(cfg, dev, heads=my_heads)
     NB = plan.NB
     rows = heads * NB
@@ -321,17 +334,21 @@ def run_ours(args):
     stream = lambda: vp(torch.cuda.current_stream().cuda_stream)
 
     stage_names = ["gather", "dense_entropy", "budget_radius", "block_mask", "sparse", "scatter"]
-    launches_per_step = 3 + 1 + 1 + 4 + 1 + 1      # block mask = vote, row scan, list fill, tile pairing
+    # block mask = vote, row scan, list fill, tile pairing; explicit layout = 3 gathers and 1 scatter
+    launches_per_step = 1 + 1 + 4 + 1 + (0 if raster else 4)
+    Qa, Ka, Va = (Qr, Kr, Vr) if raster else (Q, K, V)          # what the attention calls of the step read
+    O_step = O_raster if raster else O_tm                      # ... and write
 
     def one_step(events=None):
         def mark(i):
             if events is not None:
                 events[i].record()
         mark(0)
-        for s_, d_ in zip((Qr, Kr, Vr), (Q, K, V)):
-            api._check(lib.tra_tile_major_gather(h, ptr(s_), ptr(d_), heads, row_bytes, stream()), "gather")
+        if not raster:
+            for s_, d_ in zip((Qr, Kr, Vr), (Q, K, V)):
+                api._check(lib.tra_tile_major_gather(h, ptr(s_), ptr(d_), heads, row_bytes, stream()), "gather")
         mark(1)
-        api._check(lib.tra_entropy_attn(h, ptr(Q), ptr(K), ptr(V), ptr(O_dense), ptr(H), None, 1, heads,
+        api._check(lib.tra_entropy_attn(h, ptr(Qa), ptr(Ka), ptr(Va), ptr(O_dense), ptr(H), None, 1, heads,
                                         scale, stream()), "entropy_attn")
         mark(2)
         api._check(lib.tra_budget_radius(h, ptr(H), ptr(budget), ptr(radius), ptr(ridx), 1, heads, stream()),
@@ -340,10 +357,11 @@ def run_ours(args):
         api._check(lib.tra_build_block_mask(h, ptr(ridx), ptr(mask), ptr(row_ptr), ptr(col_idx),
                                             col_idx.numel(), ptr(nnz), ptr(pairs), 1, heads, stream()), "block_mask")
         mark(4)
-        api._check(lib.tra_sparse_attn(h, ptr(Q), ptr(K), ptr(V), ptr(row_ptr), ptr(col_idx), None, ptr(pairs),
-                                       ptr(O_tm), None, 1, heads, scale, stream()), "sparse_attn")
+        api._check(lib.tra_sparse_attn(h, ptr(Qa), ptr(Ka), ptr(Va), ptr(row_ptr), ptr(col_idx), None, ptr(pairs),
+                                       ptr(O_step), None, 1, heads, scale, stream()), "sparse_attn")
         mark(5)
-        api._check(lib.tra_tile_major_scatter(h, ptr(O_tm), ptr(O_raster), heads, row_bytes, stream()), "scatter")
+        if not raster:
+            api._check(lib.tra_tile_major_scatter(h, ptr(O_tm), ptr(O_raster), heads, row_bytes, stream()), "scatter")
         mark(6)
 
     for i in range(args.warmup):
@@ -389,7 +407,13 @@ def run_ours(args):
     peak_note = f"{peaks['_source']} bf16 sustained cuBLAS"
 
     # ---- launches timed on their own (back to back, as the sparse steps of a schedule run) -------
+    # From here on the tensors are tile-major (plan_tm): the explicit gather / scatter of the paper's design,
+    # which a raster-order step does without, is timed here.
     reps = max(2, min(5, args.steps))
+    gather_all = lambda: [plan_tm.tile_major_gather(s_, out=d_) for s_, d_ in zip((Qr, Kr, Vr), (Q, K, V))]
+    t_gather_explicit = time_ms(gather_all, reps, 1) * 1e-3
+    t_scatter_explicit = time_ms(lambda: plan_tm.tile_major_scatter(O_tm, out=O_dense), reps, 1) * 1e-3
+    plan_step, plan = plan, plan_tm
     sparse_call = lambda tp: plan.sparse_attn(Q, K, V, row_ptr, col_idx, O=O_tm, tile_pairs=tp)
     t_plain = time_ms(lambda: plan.entropy_attn(Q, K, V, O=O_dense, want_entropy=False), reps) * 1e-3
     t_sparse_b2b = time_ms(lambda: sparse_call(pairs), 2 * reps, 2) * 1e-3
@@ -398,6 +422,25 @@ def run_ours(args):
     t_token = time_ms(lambda: plan.sparse_attn(Q, K, V, row_ptr, col_idx, O=O_tm, ridx=ridx, tile_pairs=pairs),
                       reps, 2) * 1e-3
     t_token_level = time_ms(lambda: plan.sparse_attn(Q, K, V, None, None, O=O_tm, ridx=ridx), reps, 1) * 1e-3
+    # the same two launches on raster-order tensors (a TRA_ORDER_RASTER plan), where the grid allows it
+    raster_order = None
+    try:
+        plan_r = plan_step if raster else api.Plan.from_config(cfg, flags=api.TRA_ORDER_RASTER)
+        O_tmp = torch.empty_like(Qr)
+        t_r_dense = time_ms(lambda: plan_r.entropy_attn(Qr, Kr, Vr, O=O_tmp, entropy=H), reps, 1)
+        t_r_sparse = time_ms(lambda: plan_r.sparse_attn(Qr, Kr, Vr, row_ptr, col_idx, O=O_tmp, tile_pairs=pairs),
+                             reps, 2)
+        plan_r.check_status()
+        same = bool(torch.equal(O_tmp, plan_tm.tile_major_scatter(sparse_call(pairs)[0])))
+        raster_order = {"dense_entropy_ms": round(t_r_dense, 3), "sparse_ms": round(t_r_sparse, 3),
+                        "sparse_output_equals_gather_attend_scatter": same,
+                        "note": "Q, K, V read in raster order through 16-row TMA boxes, O written in raster order: "
+                                "no gather / scatter pass, slower launches"}
+        del O_tmp
+        if not raster:
+            plan_r.close()
+    except api.TraError:
+        pass
     plan.entropy_attn(Q, K, V, O=O_dense, entropy=H)      # O_dense and O_tm hold the timed pass's results again
     sparse_call(pairs)
 
@@ -420,7 +463,12 @@ def run_ours(args):
         "budget_radius_gbs": round(heads * N * 14 / (stage_ms["budget_radius"]["mean"] * 1e-3) / 1e9, 1),
         "block_mask_gbs": round((heads * N * 2 + heads * NB * NB + 4 * rows + 4 * int(nnz.item()))
                                 / (stage_ms["block_mask"]["mean"] * 1e-3) / 1e9, 2),
-        "gather_gbs": round(3 * 2 * heads * N * row_bytes / (stage_ms["gather"]["mean"] * 1e-3) / 1e9, 1),
+        "layout": "raster order read through 16-row TMA boxes (no gather / scatter pass in the step)" if raster
+                  else "explicit gather / scatter inside the step",
+        "raster_order": raster_order,
+        "explicit_gather_ms": round(t_gather_explicit * 1e3, 4),
+        "explicit_scatter_ms": round(t_scatter_explicit * 1e3, 4),
+        "gather_gbs": round(3 * 2 * heads * N * row_bytes / t_gather_explicit / 1e9, 1),
     }
 
     # `roofline` is the kernel that dominates the step (the fused dense + entropy launch, ~70 % of a
@@ -479,10 +527,13 @@ def run_ours(args):
         del q_keep, k_keep
     if extras:
         one_step()                       # every buffer holds the default pass again
+        if raster:                       # ... with tile-major Q, K, V and dense output, for the CPU sample's check
+            gather_all()
+            plan.entropy_attn(Q, K, V, O=O_dense, entropy=H)
         torch.cuda.synchronize()
 
     # ---- end to end: host buffers in, host buffer out, copies inside the timed region --------
-    e2e = run_e2e(args, api, plan, (Qr, Kr, Vr), O_raster, flops_rank, world, dev)
+    e2e = run_e2e(args, api, plan_step, (Qr, Kr, Vr), O_raster, flops_rank, world, dev)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -504,6 +555,8 @@ def run_ours(args):
         }
         print(json.dumps(line))
     plan.close()
+    if plan_step is not plan:
+        plan_step.close()
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
@@ -846,6 +899,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="the timed steps, e2e and CPU baseline only")
+    ap.add_argument("--raster", action="store_true",
+                    help="run the timed step on raster-order tensors (TRA_ORDER_RASTER plan, no gather / scatter)")
     ap.add_argument("--no-schedule", dest="schedule", action="store_false")
     ap.add_argument("--no-sweeps", dest="sweeps", action="store_false",
                     help="skip the tau / candidate-set / decay / tile-shape / block-size rows")

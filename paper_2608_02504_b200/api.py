@@ -177,25 +177,27 @@ class Plan:
         _check(self.status(stream), "tra_plan_status")
 
     # -- layout ---------------------------------------------------------------------------
-    def _permute(self, fn, src, name):
+    def _permute(self, fn, src, name, out=None):
         if not (src.is_cuda and src.is_contiguous()):
             raise ValueError(f"{name}: expected a contiguous CUDA tensor")
         if src.dim() < 2 or src.shape[-2] != self.N:
             raise ValueError(f"{name}: expected [..., N, row]")
         row_bytes = src.shape[-1] * src.element_size()
         n_bh = src.numel() // (self.N * src.shape[-1])
-        dst = torch.empty_like(src)
+        dst = torch.empty_like(src) if out is None else out
+        if not (dst.is_cuda and dst.is_contiguous() and dst.shape == src.shape and dst.dtype == src.dtype):
+            raise ValueError(f"{name}: `out` must be a contiguous CUDA tensor like the input")
         _check(fn(self._h, ctypes.c_void_p(src.data_ptr()), ctypes.c_void_p(dst.data_ptr()), n_bh,
                   row_bytes, _stream()), name)
         return dst
 
-    def tile_major_gather(self, x_raster):
-        """raster-order [..., N, row] -> tile-major order (new tensor)."""
-        return self._permute(_lib.tra_tile_major_gather, x_raster, "tra_tile_major_gather")
+    def tile_major_gather(self, x_raster, out=None):
+        """raster-order [..., N, row] -> tile-major order (a new tensor, or ``out``)."""
+        return self._permute(_lib.tra_tile_major_gather, x_raster, "tra_tile_major_gather", out)
 
-    def tile_major_scatter(self, x_tile_major):
-        """tile-major order [..., N, row] -> raster order (new tensor)."""
-        return self._permute(_lib.tra_tile_major_scatter, x_tile_major, "tra_tile_major_scatter")
+    def tile_major_scatter(self, x_tile_major, out=None):
+        """tile-major order [..., N, row] -> raster order (a new tensor, or ``out``)."""
+        return self._permute(_lib.tra_tile_major_scatter, x_tile_major, "tra_tile_major_scatter", out)
 
     # -- the four hot calls -------------------------------------------------------------
     def _bh(self, Q):

@@ -512,9 +512,13 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
   asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsControl));
   if (warp == 8) {
     // ================================================================== TMA producer
-    if (lane == 0) {
+    // One lane runs the producer; with the tensors in raster order the whole warp runs it in step (same state in
+    // every lane), so that the sixteen small boxes of a tile are issued by sixteen lanes at once.
+    const bool wide = slice_raster != nullptr;
+    if (lane == 0 || wide) {
       const uint32_t qbar = smem_u32(&ctl->q_full);
-      mbar_expect_tx(qbar, 2 * C::kQTileBytes);
+      if (lane == 0) mbar_expect_tx(qbar, 2 * C::kQTileBytes);
+      if (wide) __syncwarp();
       // Rows [row0, row0 + rows) of the tile-major order into a tile at `dst` (atoms `atom_bytes` apart).  With the
       // tensors in tile-major order that is one box per 64-column atom.  With the tensors in RASTER order
       // (slice_raster != NULL) every 16 consecutive tile-major positions are 16 consecutive raster rows, which
@@ -524,14 +528,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         if (slice_raster == nullptr) {
           for (int a = 0; a < C::kAtoms; ++a) tma_load_3d(dst + a * atom_bytes, map, bar, a * 64, row0, bh);
         } else {
-          int rr[kTileM / 16];
-#pragma unroll
-          for (int j = 0; j < kTileM / 16; ++j) rr[j] = j * 16 < rows ? __ldg(slice_raster + (row0 >> 4) + j) : 0;
-#pragma unroll
-          for (int j = 0; j < kTileM / 16; ++j)
-            if (j * 16 < rows)
-              for (int a = 0; a < C::kAtoms; ++a)
-                tma_load_3d(dst + a * atom_bytes + j * 2048, map, bar, a * 64, rr[j], bh);
+          const int j = lane & 7, a = lane >> 3;           // lane -> (slice, atom)
+          if (a < C::kAtoms && j * 16 < rows)
+            tma_load_3d(dst + a * atom_bytes + j * 2048, map, bar, a * 64, __ldg(slice_raster + (row0 >> 4) + j), bh);
         }
       };
       for (int k = 0; k < 2; ++k)      // a missing tile loads rows nobody uses
@@ -540,7 +539,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       bool alive = true;
       auto load_tile = [&](const CUtensorMap* map, int slot, int v) {
         const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
-        mbar_expect_tx(fbar, C::kSlotBytes);
+        if (lane == 0) mbar_expect_tx(fbar, C::kSlotBytes);
+        if (wide) __syncwarp();
         load_rows(map, smem_u32(sKV + slot * C::kSlotBytes), fbar, v * blk, BN, C::kKVAtomBytes);
       };
       if constexpr (kDense) {
@@ -631,7 +631,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           }
         }
 #ifdef TRA_DEBUG
-        ctl->dbg_jobs[3] = (int)ks.jobs - (ks.e == vs.e ? 0 : 1 << 20);     // both streams walked every entry
+        if (lane == 0) ctl->dbg_jobs[3] = (int)ks.jobs - (ks.e == vs.e ? 0 : 1 << 20);     // both streams walked every entry
 #endif
       }
     }
