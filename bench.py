@@ -294,20 +294,27 @@ def run_ours(args):
 
     sampler = make_sampler(local)
     sampler.start()                     # started early; only samples of the timed region count
-    # The timed step gathers Q, K, V into tile-major order and scatters O back, as the paper does.  With
-    # --raster (and a grid that allows it) the step runs on the raster-order tensors instead: the kernels fetch
-    # 16-token runs through TMA boxes of their own and there is no gather / scatter pass.  That saves the two
-    # layout passes and costs more in the attention launches (sixteen small boxes per tile instead of two), so it
-    # is not the default; `stages.raster_order` has both launches' times either way.  plan_tm is the plan for
+    # Layout of the timed step (the caller's tensors are in raster order):
+    #   "qo" (default where the grid allows it): a TRA_ORDER_RASTER_QO plan.  K and V are gathered into tile-major
+    #        order; Q is read and O written in raster order by the attention launches themselves (Q is loaded
+    #        once per thread block and O rows are stored one by one anyway), so the gather of Q and the scatter
+    #        of O drop out at no cost to the launches;
+    #   "explicit": gather Q, K, V and scatter O, as the paper does;
+    #   "raster": a TRA_ORDER_RASTER plan, no layout pass at all; K / V tiles then arrive as sixteen small TMA
+    #        boxes instead of two, which costs the launches more than the passes it saves.
+    # `stages.raster_order` has the launch times of the third form whatever the choice.  plan_tm is the plan for
     # tile-major tensors, which the measurements after the timed region use.
     plan_tm = api.Plan.from_config(cfg)
-    plan, raster = plan_tm, False
-    if args.raster:
+    plan, layout = plan_tm, "explicit"
+    if args.layout != "explicit":
         try:
-            plan = api.Plan.from_config(cfg, flags=api.TRA_ORDER_RASTER)
-            raster = True
+            plan = api.Plan.from_config(cfg, flags=api.TRA_ORDER_RASTER if args.layout == "raster"
+                                        else api.TRA_ORDER_RASTER_QO)
+            layout = args.layout
         except api.TraError:
             pass
+    raster = layout == "raster"             # K and V in raster order too
+    raster_qo = layout != "explicit"        # Q and O in raster order
     Qr, Kr, Vr = workloads.make_qkv(cfg, dev, heads=my_heads)
     NB = plan.NB
     rows = heads * NB
@@ -335,18 +342,19 @@ def run_ours(args):
 
     stage_names = ["gather", "dense_entropy", "budget_radius", "block_mask", "sparse", "scatter"]
     # block mask = vote, row scan, list fill, tile pairing; explicit layout = 3 gathers and 1 scatter
-    launches_per_step = 1 + 1 + 4 + 1 + (0 if raster else 4)
-    Qa, Ka, Va = (Qr, Kr, Vr) if raster else (Q, K, V)          # what the attention calls of the step read
-    O_step = O_raster if raster else O_tm                      # ... and write
+    launches_per_step = 1 + 1 + 4 + 1 + (0 if raster else (2 if raster_qo else 4))
+    Qa = Qr if raster_qo else Q                                # what the attention calls of the step read
+    Ka, Va = (Kr, Vr) if raster else (K, V)
+    O_step = O_raster if raster_qo else O_tm                   # ... and write
+    to_gather = [] if raster else ([(Kr, K), (Vr, V)] if raster_qo else [(Qr, Q), (Kr, K), (Vr, V)])
 
     def one_step(events=None):
         def mark(i):
             if events is not None:
                 events[i].record()
         mark(0)
-        if not raster:
-            for s_, d_ in zip((Qr, Kr, Vr), (Q, K, V)):
-                api._check(lib.tra_tile_major_gather(h, ptr(s_), ptr(d_), heads, row_bytes, stream()), "gather")
+        for s_, d_ in to_gather:
+            api._check(lib.tra_tile_major_gather(h, ptr(s_), ptr(d_), heads, row_bytes, stream()), "gather")
         mark(1)
         api._check(lib.tra_entropy_attn(h, ptr(Qa), ptr(Ka), ptr(Va), ptr(O_dense), ptr(H), None, 1, heads,
                                         scale, stream()), "entropy_attn")
@@ -360,7 +368,7 @@ def run_ours(args):
         api._check(lib.tra_sparse_attn(h, ptr(Qa), ptr(Ka), ptr(Va), ptr(row_ptr), ptr(col_idx), None, ptr(pairs),
                                        ptr(O_step), None, 1, heads, scale, stream()), "sparse_attn")
         mark(5)
-        if not raster:
+        if not raster_qo:
             api._check(lib.tra_tile_major_scatter(h, ptr(O_tm), ptr(O_raster), heads, row_bytes, stream()), "scatter")
         mark(6)
 
@@ -463,8 +471,11 @@ def run_ours(args):
         "budget_radius_gbs": round(heads * N * 14 / (stage_ms["budget_radius"]["mean"] * 1e-3) / 1e9, 1),
         "block_mask_gbs": round((heads * N * 2 + heads * NB * NB + 4 * rows + 4 * int(nnz.item()))
                                 / (stage_ms["block_mask"]["mean"] * 1e-3) / 1e9, 2),
-        "layout": "raster order read through 16-row TMA boxes (no gather / scatter pass in the step)" if raster
-                  else "explicit gather / scatter inside the step",
+        "layout": {"qo": "K and V gathered into tile-major order inside the step; Q read and O written in raster "
+                         "order by the attention launches (no gather of Q, no scatter of O)",
+                   "explicit": "Q, K, V gathered and O scattered inside the step",
+                   "raster": "Q, K, V read and O written in raster order by the attention launches (16-row TMA "
+                             "boxes; no gather / scatter pass)"}[layout],
         "raster_order": raster_order,
         "explicit_gather_ms": round(t_gather_explicit * 1e3, 4),
         "explicit_scatter_ms": round(t_scatter_explicit * 1e3, 4),
@@ -527,7 +538,7 @@ def run_ours(args):
         del q_keep, k_keep
     if extras:
         one_step()                       # every buffer holds the default pass again
-        if raster:                       # ... with tile-major Q, K, V and dense output, for the CPU sample's check
+        if raster_qo:                    # ... with tile-major Q, K, V and dense output, for the CPU sample's check
             gather_all()
             plan.entropy_attn(Q, K, V, O=O_dense, entropy=H)
         torch.cuda.synchronize()
@@ -899,8 +910,9 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=8192)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="the timed steps, e2e and CPU baseline only")
-    ap.add_argument("--raster", action="store_true",
-                    help="run the timed step on raster-order tensors (TRA_ORDER_RASTER plan, no gather / scatter)")
+    ap.add_argument("--layout", default="qo", choices=["qo", "explicit", "raster"],
+                    help="which tensors the attention launches of the timed step take in raster order: Q and O "
+                         "(default), none (explicit gather / scatter), or all")
     ap.add_argument("--no-schedule", dest="schedule", action="store_false")
     ap.add_argument("--no-sweeps", dest="sweeps", action="store_false",
                     help="skip the tau / candidate-set / decay / tile-shape / block-size rows")

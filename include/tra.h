@@ -15,7 +15,8 @@
  * `block` consecutive tile-major positions (Algorithm 1: q = u*b + i, q < N);
  * NB = ceil(N / block).  tra_tile_major_gather / _scatter move tensors between
  * raster order (n = (t*H + y)*W + x) and tile-major order.  A plan created with
- * TRA_ORDER_RASTER takes Q, K, V and O in raster order instead and needs no such pass.
+ * TRA_ORDER_RASTER takes Q, K, V and O in raster order instead and needs no such pass
+ * (TRA_ORDER_RASTER_QO: Q and O only).
  *
  * Joint text-video attention (Section 3.2, last paragraph; Algorithm 1).  With cfg.n_text > 0 a
  * sequence is the N video tokens followed by n_text text tokens, S = N + n_text; S takes the place
@@ -61,6 +62,11 @@ extern "C" {
                              /* the mask stay in tile-major order: they only travel between this library's    */
                              /* calls.  Needs W, tile_w and block to be multiples of 16 (else                  */
                              /* tra_plan_create returns TRA_ERR_UNSUPPORTED).                                 */
+#define TRA_ORDER_RASTER_QO 4u /* only Q and O are in raster order; K and V are tile-major (gathered by the     */
+                               /* caller).  Q is loaded once per thread block and O rows are stored one by one */
+                               /* anyway, so this costs nothing in the launches and saves the gather of Q and  */
+                               /* the scatter of O; the many K / V tile loads keep their two large boxes.      */
+                               /* Same conditions as TRA_ORDER_RASTER, which takes precedence.                 */
 
 /* entropy-to-budget maps */
 #define TRA_BUDGET_UNIFORM 0   /* K = ceil(tau exp(H)): the uniform-support map of Eq. 8 (the paper's choice) */
@@ -86,7 +92,7 @@ typedef struct {
                        /* one must reach full support (may be +inf).  NULL = radius_policy       */
   int n_radii;
   int radius_policy;   /* TRA_RADII_* (used when radii == NULL)                                  */
-  unsigned flags;      /* TRA_KEEP_DIAGONAL | TRA_ORDER_RASTER                                   */
+  unsigned flags;      /* TRA_KEEP_DIAGONAL | TRA_ORDER_RASTER | TRA_ORDER_RASTER_QO             */
   int budget_map;      /* TRA_BUDGET_* used by tra_budget_radius                                 */
   int n_text;          /* text tokens that follow the video tokens in every sequence (>= 0)     */
 } tra_config_t;

@@ -20,6 +20,7 @@ TRA_OK = 0
 TRA_ERR_INVALID_ARG, TRA_ERR_UNSUPPORTED, TRA_ERR_CAPACITY, TRA_ERR_CUDA, TRA_ERR_TIMEOUT, TRA_ERR_BOUNDS = -1, -2, -3, -4, -5, -6
 TRA_KEEP_DIAGONAL = 1
 TRA_ORDER_RASTER = 2
+TRA_ORDER_RASTER_QO = 4
 TRA_RADII_EXTENDED = 0
 TRA_RADII_LITERAL = 1
 TRA_BUDGET_UNIFORM = 0
@@ -336,8 +337,8 @@ class HostPipeline:
         self.workspace = torch.empty(self.workspace_bytes + 256, dtype=torch.uint8, device=self.dev)
         self._ws_ptr = (self.workspace.data_ptr() + 255) & ~255
         # 3 gathers, dense, budget, vote + scan + fill + pairing, sparse, scatter; a raster-order plan has no
-        # gathers and no scatter
-        self.launches_per_group = 7 if plan.flags & TRA_ORDER_RASTER else 11
+        # gathers and no scatter, one with only Q and O in raster order gathers K and V
+        self.launches_per_group = 7 if plan.flags & TRA_ORDER_RASTER else (9 if plan.flags & TRA_ORDER_RASTER_QO else 11)
         self.n_groups = len(self.group_sizes(heads, self.group, self.first_group))
 
     @staticmethod

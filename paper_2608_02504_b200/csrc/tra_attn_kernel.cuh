@@ -367,7 +367,7 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
                 const int32_t* __restrict__ row_ptr, const int32_t* __restrict__ col_idx,
                 const int32_t* __restrict__ tile_pairs, int N, int NB, float scale_log2,
                 int* __restrict__ status, TokenMaskArgs tm, int blk_arg,
-                const int32_t* __restrict__ slice_raster) {
+                const int32_t* __restrict__ slice_raster, int raster_kv) {
   using C = Cfg<D, BN>;
   static_assert(!(kAny && kTokenMask), "the token mask needs blocks of whole 16-key slices");
   // kAny: blocks of blk <= BN tokens (BN = blk rounded up to a multiple of 16).  A key tile is still BN rows,
@@ -514,7 +514,8 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
     // ================================================================== TMA producer
     // One lane runs the producer; with the tensors in raster order the whole warp runs it in step (same state in
     // every lane), so that the sixteen small boxes of a tile are issued by sixteen lanes at once.
-    const bool wide = slice_raster != nullptr;
+    // (slice_raster is set when Q and O are in raster order; raster_kv tells whether K and V are as well)
+    const bool wide = slice_raster != nullptr && raster_kv;
     if (lane == 0 || wide) {
       const uint32_t qbar = smem_u32(&ctl->q_full);
       if (lane == 0) mbar_expect_tx(qbar, 2 * C::kQTileBytes);
@@ -524,24 +525,30 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
       // (slice_raster != NULL) every 16 consecutive tile-major positions are 16 consecutive raster rows, which
       // start at slice_raster[position / 16]: one box of 16 rows per slice, 2 KB apart in the tile (the swizzle
       // pattern repeats every 8 rows, so the tile in shared memory is the same either way).
-      auto load_rows = [&](const CUtensorMap* map, uint32_t dst, uint32_t bar, int row0, int rows, int atom_bytes) {
-        if (slice_raster == nullptr) {
-          for (int a = 0; a < C::kAtoms; ++a) tma_load_3d(dst + a * atom_bytes, map, bar, a * 64, row0, bh);
-        } else {
+      auto load_rows = [&](const CUtensorMap* map, uint32_t dst, uint32_t bar, int row0, int rows, int atom_bytes,
+                           bool by_runs) {
+        if (!by_runs) {
+          if (lane == 0)
+            for (int a = 0; a < C::kAtoms; ++a) tma_load_3d(dst + a * atom_bytes, map, bar, a * 64, row0, bh);
+        } else if (wide) {
           const int j = lane & 7, a = lane >> 3;           // lane -> (slice, atom)
           if (a < C::kAtoms && j * 16 < rows)
             tma_load_3d(dst + a * atom_bytes + j * 2048, map, bar, a * 64, __ldg(slice_raster + (row0 >> 4) + j), bh);
+        } else {                                           // the one producer lane issues every box (Q only)
+          for (int j = 0; j * 16 < rows; ++j)
+            for (int a = 0; a < C::kAtoms; ++a)
+              tma_load_3d(dst + a * atom_bytes + j * 2048, map, bar, a * 64, __ldg(slice_raster + (row0 >> 4) + j), bh);
         }
       };
       for (int k = 0; k < 2; ++k)      // a missing tile loads rows nobody uses
         load_rows(&map_q, smem_u32(sQ + k * C::kQTileBytes), qbar, max(tile_index(k), 0) * tile_rows, kTileM,
-                  C::kQAtomBytes);
+                  C::kQAtomBytes, slice_raster != nullptr);
       bool alive = true;
       auto load_tile = [&](const CUtensorMap* map, int slot, int v) {
         const uint32_t fbar = smem_u32(&ctl->kv_full[slot]);
         if (lane == 0) mbar_expect_tx(fbar, C::kSlotBytes);
         if (wide) __syncwarp();
-        load_rows(map, smem_u32(sKV + slot * C::kSlotBytes), fbar, v * blk, BN, C::kKVAtomBytes);
+        load_rows(map, smem_u32(sKV + slot * C::kSlotBytes), fbar, v * blk, BN, C::kKVAtomBytes, wide);
       };
       if constexpr (kDense) {
         // Loads go K0, V0, K1, V1, ... into consecutive slots.  The MMA warp hands slots back in
@@ -1231,11 +1238,13 @@ int launch(const tra_attn_args& a) {
   const tra_plan_t* plan = a.plan;
   CUtensorMap mq, mk, mv;
   int rc;
-  const int32_t* slice_raster = (plan->cfg.flags & TRA_ORDER_RASTER) ? plan->d_slice_raster : nullptr;
+  const bool raster_kv = (plan->cfg.flags & TRA_ORDER_RASTER) != 0;
+  const int32_t* slice_raster = (plan->cfg.flags & (TRA_ORDER_RASTER | TRA_ORDER_RASTER_QO)) ? plan->d_slice_raster
+                                                                                              : nullptr;
   // boxes: a whole tile per 64-column atom, or (raster order) one 16-token run
   if ((rc = make_map(&mq, a.Q, D, plan->S, a.BH, slice_raster ? 16 : kTileM)) != TRA_OK) return rc;
-  if ((rc = make_map(&mk, a.K, D, plan->S, a.BH, slice_raster ? 16 : BN)) != TRA_OK) return rc;
-  if ((rc = make_map(&mv, a.V, D, plan->S, a.BH, slice_raster ? 16 : BN)) != TRA_OK) return rc;
+  if ((rc = make_map(&mk, a.K, D, plan->S, a.BH, raster_kv ? 16 : BN)) != TRA_OK) return rc;
+  if ((rc = make_map(&mv, a.V, D, plan->S, a.BH, raster_kv ? 16 : BN)) != TRA_OK) return rc;
   auto kern = tra_attn_kernel<D, BN, kEntropy, kTokenMask, kDense, kLse, kAny>;
   TokenMaskArgs tm = {plan->d_boxes, plan->d_slice, plan->d_coord_packed, plan->d_theta, a.ridx,
                       plan->N,       plan->cfg.T,   plan->n_radii};
@@ -1246,7 +1255,7 @@ int launch(const tra_attn_args& a) {
   kern<<<grid, kThreads, C::kSmemBytes, a.stream>>>(mq, mk, mv, (__nv_bfloat16*)a.O, a.entropy, a.lse, a.row_ptr,
                                                     a.col_idx, a.tile_pairs, plan->S, plan->NB,
                                                     a.sm_scale * kLog2e, plan->d_status, tm, plan->cfg.block,
-                                                    slice_raster);
+                                                    slice_raster, raster_kv ? 1 : 0);
   TRA_CUDA_CHECK(cudaGetLastError());
   return TRA_OK;
 }

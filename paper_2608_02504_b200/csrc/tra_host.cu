@@ -144,17 +144,19 @@ extern "C" int tra_hot_path_host(tra_plan_t* plan, const void* Q_host, const voi
     TRA_CUDA_CHECK(cudaStreamWaitEvent(cs, ready, 0));
     // the pass itself; a raster-order plan reads the staging buffers in place and writes O into the output
     // staging buffer, so the gather and scatter kernels drop out
-    const bool raster = (plan->cfg.flags & TRA_ORDER_RASTER) != 0;
+    // (with TRA_ORDER_RASTER_QO that holds for Q and O; K and V are still gathered)
+    const bool raster_kv = (plan->cfg.flags & TRA_ORDER_RASTER) != 0;
+    const bool raster = raster_kv || (plan->cfg.flags & TRA_ORDER_RASTER_QO) != 0;      // Q and O
     int rc;
+    for (int t = raster ? 1 : 0; t < 3 && !raster_kv; ++t)
+      if ((rc = tra_tile_major_gather(plan, ws + L.stage_in[b][t], ws + L.qkv[t], n, row_bytes, cs)) != TRA_OK)
+        return rc;
     if (!raster) {
-      for (int t = 0; t < 3; ++t)
-        if ((rc = tra_tile_major_gather(plan, ws + L.stage_in[b][t], ws + L.qkv[t], n, row_bytes, cs)) != TRA_OK)
-          return rc;
       if (!(in_free[b] = pool.make())) return TRA_ERR_CUDA;
       TRA_CUDA_CHECK(cudaEventRecord(in_free[b], cs));
     }
-    const void *Q = ws + (raster ? L.stage_in[b][0] : L.qkv[0]), *K = ws + (raster ? L.stage_in[b][1] : L.qkv[1]),
-               *V = ws + (raster ? L.stage_in[b][2] : L.qkv[2]);
+    const void *Q = ws + (raster ? L.stage_in[b][0] : L.qkv[0]), *K = ws + (raster_kv ? L.stage_in[b][1] : L.qkv[1]),
+               *V = ws + (raster_kv ? L.stage_in[b][2] : L.qkv[2]);
     if ((rc = tra_entropy_attn(plan, Q, K, V, ws + L.o_dense, (float*)(ws + L.entropy), nullptr, 1, n, sm_scale,
                                cs)) != TRA_OK)
       return rc;

@@ -301,12 +301,12 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
     for (size_t i = 0; i < n; ++i) field_pos[i] = (uint16_t)(pos_of[per * i] / per);
   }
 
-  // Raster-order attention (TRA_ORDER_RASTER): the raster row at which every run of 16 consecutive tile-major
+  // Raster-order attention (TRA_ORDER_RASTER, TRA_ORDER_RASTER_QO): the raster row at which every run of 16 consecutive tile-major
   // positions starts.  Needs every such run to be 16 consecutive raster rows (W and the tile width multiples of
   // 16) and blocks that start on run boundaries; entries past the sequence hold S, a row outside the tensor (the
   // load of such a run is filled with zeros).
   std::vector<int32_t> slice_raster;
-  if (cfg->flags & TRA_ORDER_RASTER) {
+  if (cfg->flags & (TRA_ORDER_RASTER | TRA_ORDER_RASTER_QO)) {
     bool runs = cfg->block % 16 == 0 && p->N % 16 == 0;
     for (int s0 = 0; s0 < p->N && runs; s0 += 16)
       for (int i = 1; i < 16 && runs; ++i) runs = raster[s0 + i] == raster[s0] + i;

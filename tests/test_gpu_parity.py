@@ -978,17 +978,26 @@ def test_raster_order_plan_equals_gather_attend_scatter(name, cfg, n_text):
             M_t, _ = plan_t.sparse_attn(Q, K, V, rp, ci, ridx=ridx)
             M_r, _ = plan_r.sparse_attn(Qr, Kr, Vr, rp, ci, ridx=ridx)
             assert torch.equal(M_r, plan_t.tile_major_scatter(M_t))
-    # the host pipeline of a raster-order plan: no gather, no scatter, same bits
+    # only Q and O in raster order (TRA_ORDER_RASTER_QO): K and V tile-major
+    plan_q = make_plan(cfg, n_text=n_text, flags=api().TRA_ORDER_RASTER_QO)
+    O_q, H_q, lse_q = plan_q.entropy_attn(Qr, K, V, want_lse=True)
+    assert torch.equal(O_q, O_r) and torch.equal(H_q, H_t) and torch.equal(lse_q, lse_t)
+    S_q, sl_q = plan_q.sparse_attn(Qr, K, V, row_ptr, col_idx, tile_pairs=pairs, want_lse=True)
+    assert torch.equal(S_q, S_r) and torch.equal(sl_q, sl_t)
+    if token_mask:
+        M_q, _ = plan_q.sparse_attn(Qr, K, V, row_ptr, col_idx, ridx=ridx)
+        assert torch.equal(M_q, plan_t.tile_major_scatter(plan_t.sparse_attn(Q, K, V, row_ptr, col_idx, ridx=ridx)[0]))
+    # the host pipelines of such plans: no gather and no scatter (7 kernels per group), or two gathers (9)
     host = [t.cpu().pin_memory() for t in (Qr, Kr, Vr)]
-    out = torch.zeros(S_r.shape, dtype=torch.bfloat16).pin_memory()
-    pipe = api().HostPipeline(plan_r, cfg["heads"], group=1)
-    assert pipe.run(host[0], host[1], host[2], out) == 7 * cfg["heads"]
-    torch.cuda.synchronize()
-    assert torch.equal(out, S_r.cpu())
-    plan_t.check_status()
-    plan_r.check_status()
-    plan_t.close()
-    plan_r.close()
+    for p_, n_launch in ((plan_r, 7), (plan_q, 9)):
+        out = torch.zeros(S_r.shape, dtype=torch.bfloat16).pin_memory()
+        pipe = api().HostPipeline(p_, cfg["heads"], group=1)
+        assert pipe.run(host[0], host[1], host[2], out) == n_launch * cfg["heads"]
+        torch.cuda.synchronize()
+        assert torch.equal(out, S_r.cpu())
+    for p_ in (plan_t, plan_r, plan_q):
+        p_.check_status()
+        p_.close()
 
 
 def test_raster_order_needs_runs_of_sixteen():
