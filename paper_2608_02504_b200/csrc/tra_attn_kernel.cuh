@@ -920,6 +920,9 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
           job_prev = job;
           if (C::kGroups > 1) active = (own_bits & low) != 0;
         }
+        // rows of the tile past its query blocks (kAny) hold no query: no exponentials for them (a warp made of such
+        // rows only keeps up with the barriers and writes zeros)
+        if (kAny && r >= tile_rows) active = false;
         const int col_limit = min(blk, N - v * blk);
         const uint32_t t_s = tmem + lane_base + buf * 128;
 
@@ -939,13 +942,15 @@ tra_attn_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant
         for (int c = 1; c < C::kChunks; ++c) reg_fence32(&sb[c * 32]);
 
         // Columns >= col_limit do not exist: the ragged last key block, and with kAny the tail of every key tile
-        // (rows of the next block, and tensor-memory columns past BN that no MMA wrote).  Only the last 32
-        // columns can be concerned unless the block is the ragged last one.
+        // (rows of the next block, and tensor-memory columns past BN that no MMA wrote).  Only the last 16
+        // columns of the tile, and those past BN, can be concerned unless the block is the ragged last one.
         if (col_limit < C::kCols) {
-          if (col_limit >= C::kCols - 32) {
+          if (col_limit > BN - 16) {        // the usual case with kAny: the block ends in the last 16 rows of the tile
 #pragma unroll
-            for (int j = C::kCols - 32; j < C::kCols; ++j)
+            for (int j = BN - 16; j < BN; ++j)
               if (j >= col_limit) sb[j] = __float_as_uint(-1e30f);
+#pragma unroll
+            for (int j = BN; j < C::kCols; ++j) sb[j] = __float_as_uint(-1e30f);
           } else {
 #pragma unroll
             for (int j = 0; j < C::kCols; ++j)
