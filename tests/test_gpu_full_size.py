@@ -99,11 +99,13 @@ BENCH_VARIANTS = [
     ("hunyuan-720p", dict(gamma=0.0513), 0, (0, 23)),
     ("wan14b-720p", dict(tile_h=1, tile_w=80), 0, (3, 30)),
     ("wan14b-720p", dict(), 256, (1, 17)),
+    ("wan14b-720p", dict(block=90, tile_h=9, tile_w=10), 0, (2, 33)),      # the paper's 90-token tiles as blocks
+    ("wan14b-720p", dict(block=120, tile_h=15, tile_w=8), 0, (4, 28)),
 ]
 
 
 @pytest.mark.parametrize("name,override,n_text,heads", BENCH_VARIANTS,
-                         ids=["tau0.5", "tau0.3", "hunyuan-gamma0.0513", "tile1x80", "text256"])
+                         ids=["tau0.5", "tau0.3", "hunyuan-gamma0.0513", "tile1x80", "text256", "block90", "block120"])
 def test_benchmark_configurations_sampled_rows(name, override, n_text, heads):
     """The configurations the benchmark times besides the default one, at full size on two heads:
     sampled rows of dense attention + entropy, the integer stages of their block rows, and the
@@ -124,7 +126,7 @@ def test_benchmark_configurations_sampled_rows(name, override, n_text, heads):
     Os2, _ = plan.sparse_attn(Q, K, V, row_ptr, col_idx)                 # consecutive tiles: the same bits
     plan.check_status()
     assert torch.equal(Os, Os2)
-    _assert_perfect_matching(pairs, len(heads), (S + 127) // 128)
+    _assert_perfect_matching(pairs, len(heads), (NB + 1) // 2 if b <= 64 else NB)      # query tiles: two small blocks or one
     rng = np.random.default_rng(19)
     worst = {"max_abs": 0.0, "n_over_atol": 0, "n": 0}
     for i in range(len(heads)):
