@@ -42,13 +42,14 @@ __device__ __forceinline__ const uint32_t* tra_count_row(const RadiusArgs& a, ui
   return a.counts + ((size_t)(tra_coord_t(c) * a.H + tra_coord_y(c)) * a.W + tra_coord_x(c)) * a.n_radii;
 }
 
-// Candidate sets of up to 128 radii (the built-in sets have about 110): the search takes two rounds
-// of independent loads instead of seven dependent ones.  Round 1 reads the token's row of the coarse
-// table (every eighth entry of its count-table row, 64 bytes, four 16-byte loads) and counts the
-// entries below the budget, which names the group of eight that holds the answer; round 2 reads
-// that group (one aligned 32-byte sector of a copy of the count table with rows padded to 128
-// entries; the rows of the table itself are not sector-aligned) and counts again.  Rows are non-decreasing, so "entries below the budget" is the index
-// of the first entry that reaches it (Eq. 14).
+// Candidate sets of up to 128 radii (the built-in sets have about 110): the search takes two steps
+// of independent loads instead of seven dependent ones.  The first reads the token's row of the
+// coarse table (every eighth entry of its count-table row, 64 bytes, four 16-byte loads) and counts
+// the entries below the budget, which names the group of eight that holds the answer; the second
+// reads that group (one aligned 32-byte sector of a copy of the count table with rows padded to 128
+// entries; the rows of the table itself are not sector-aligned) and counts again.  Rows are
+// non-decreasing, so "entries below the budget" is the index of the first entry that reaches it
+// (Eq. 14).
 __global__ void __launch_bounds__(256) tra_budget_radius_2round_kernel(RadiusArgs a, const uint32_t* __restrict__ coarse) {
   const long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= a.total) return;
