@@ -524,7 +524,9 @@ tra_col_idx_fill_kernel(const uint8_t* __restrict__ block_mask, const int32_t* _
 // v = -1 for a lone tile.
 // Any perfect matching gives the same attention output; the choice only moves time.
 // ---------------------------------------------------------------------------------------
+#ifndef TRA_PAIR_WINDOW
 #define TRA_PAIR_WINDOW 8
+#endif
 #define TRA_PAIR_CANDS (TRA_PAIR_WINDOW + 3)
 #define TRA_PAIR_CHUNK 32
 #define TRA_PAIR_THREADS 512

@@ -134,6 +134,7 @@ extern "C" int tra_plan_create(tra_plan_t** out, const tra_config_t* cfg, void* 
   if (cfg->budget_map != TRA_BUDGET_UNIFORM && cfg->budget_map != TRA_BUDGET_LOGNORMAL)
     return TRA_ERR_INVALID_ARG;
   if (cfg->n_text < 0 || cfg->n_text > (1 << 24)) return TRA_ERR_INVALID_ARG;
+  if (cfg->flags & ~(TRA_KEEP_DIAGONAL | TRA_ORDER_RASTER | TRA_ORDER_RASTER_QO)) return TRA_ERR_INVALID_ARG;
 
   tra_plan* p = new tra_plan();
   memset(p, 0, sizeof(*p));

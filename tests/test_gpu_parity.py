@@ -61,6 +61,7 @@ def test_plan_tables_bit_exact(cfg, policy):
 def test_plan_rejects_bad_arguments():
     a = api()
     for kw in (dict(head_dim=96), dict(block=8), dict(tau=0.0), dict(gamma=-1.0), dict(T=0),
+               dict(flags=8),                         # an unknown flag
                dict(radii=[0.0, 1.0, 2.0]),          # last candidate does not reach full support
                dict(radii=[0.0, 2.0, 1.0, 1e9])):    # not ascending
         with pytest.raises(a.TraError):
