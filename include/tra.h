@@ -113,6 +113,8 @@ int tra_plan_num_tokens(const tra_plan_t* plan);   /* S = N + n_text: tokens per
 int tra_plan_num_video_tokens(const tra_plan_t* plan); /* N = T*H*W */
 int tra_plan_num_blocks(const tra_plan_t* plan);   /* NB */
 int tra_plan_num_radii(const tra_plan_t* plan);    /* |R| */
+int tra_plan_num_tile_pairs(const tra_plan_t* plan); /* entries per (batch, head) of the tile-pair table of
+                                                        tra_build_block_mask: ceil(NT / 2); 0 for blocks <= 32 */
 /* Copies plan tables to HOST buffers (synchronises): radii[|R|] (double), theta[|R|*T]
  * (int32, theta[k*T + delta]), coord[N*3] (int32 t,y,x per tile-major position).  Any may be NULL. */
 int tra_plan_tables(const tra_plan_t* plan, double* radii, int32_t* theta, int32_t* coord);

@@ -28,7 +28,7 @@ TRA_BUDGET_LOGNORMAL = 1
 
 EXPORTS = [
     "tra_plan_create", "tra_plan_destroy", "tra_plan_num_tokens", "tra_plan_num_video_tokens", "tra_plan_num_blocks",
-    "tra_plan_num_radii", "tra_plan_tables", "tra_plan_count_table", "tra_plan_status",
+    "tra_plan_num_radii", "tra_plan_num_tile_pairs", "tra_plan_tables", "tra_plan_count_table", "tra_plan_status",
     "tra_status_string", "tra_selftest_wait_timeout", "tra_tile_major_gather", "tra_tile_major_scatter",
     "tra_entropy_attn", "tra_budget_radius", "tra_build_block_mask", "tra_sparse_attn",
     "tra_build_block_list_static",
@@ -57,7 +57,8 @@ def _load():
     vp, i32, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
     lib.tra_plan_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(tra_config_t), vp]
     lib.tra_plan_destroy.argtypes = [vp]
-    for name in ("tra_plan_num_tokens", "tra_plan_num_video_tokens", "tra_plan_num_blocks", "tra_plan_num_radii"):
+    for name in ("tra_plan_num_tokens", "tra_plan_num_video_tokens", "tra_plan_num_blocks", "tra_plan_num_radii",
+                 "tra_plan_num_tile_pairs"):
         getattr(lib, name).argtypes = [vp]
     lib.tra_plan_tables.argtypes = [vp, vp, vp, vp]
     lib.tra_plan_count_table.argtypes = [vp, vp]
@@ -246,8 +247,7 @@ class Plan:
     def n_tile_pairs(self):
         """Thread blocks per (batch, head) of a block-sparse launch: pairs of query tiles (a tile holds two
         blocks of up to 64 tokens, or one larger block)."""
-        per_tile = 2 if self.block <= 64 else 1
-        return ((self.NB + per_tile - 1) // per_tile + 1) // 2
+        return _lib.tra_plan_num_tile_pairs(self._h)
 
     def build_block_mask(self, ridx, block_mask=None, row_ptr=None, col_idx=None, nnz=None, tile_pairs=None,
                          want_tile_pairs=False):
@@ -266,7 +266,8 @@ class Plan:
         if nnz is None:
             nnz = torch.zeros(1, dtype=torch.int64, device=dev)
         if tile_pairs is None and want_tile_pairs:
-            tile_pairs = torch.empty(B * heads, self.n_tile_pairs, 2, dtype=torch.int32, device=dev)
+            # (blocks of 32 tokens or fewer have no tile pairs: one entry, so that the library's refusal is seen)
+            tile_pairs = torch.empty(B * heads, max(self.n_tile_pairs, 1), 2, dtype=torch.int32, device=dev)
         _check(_lib.tra_build_block_mask(self._h, _dev(ridx, torch.int16, "ridx"),
                                          _dev(block_mask, torch.uint8, "block_mask"),
                                          _dev(row_ptr, torch.int32, "row_ptr"),

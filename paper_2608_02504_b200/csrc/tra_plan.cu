@@ -382,6 +382,12 @@ extern "C" int tra_plan_num_tokens(const tra_plan_t* plan) { return plan ? plan-
 extern "C" int tra_plan_num_video_tokens(const tra_plan_t* plan) { return plan ? plan->N : TRA_ERR_INVALID_ARG; }
 extern "C" int tra_plan_num_blocks(const tra_plan_t* plan) { return plan ? plan->NB : TRA_ERR_INVALID_ARG; }
 extern "C" int tra_plan_num_radii(const tra_plan_t* plan) { return plan ? plan->n_radii : TRA_ERR_INVALID_ARG; }
+extern "C" int tra_plan_num_tile_pairs(const tra_plan_t* plan) {
+  if (!plan) return TRA_ERR_INVALID_ARG;
+  if (plan->cfg.block <= 32) return 0;                 // no attention launch for such blocks
+  const int G = tra_blocks_per_tile(plan->cfg.block);
+  return ((plan->NB + G - 1) / G + 1) / 2;
+}
 
 extern "C" int tra_plan_tables(const tra_plan_t* plan, double* radii, int32_t* theta, int32_t* coord) {
   if (!plan) return TRA_ERR_INVALID_ARG;
